@@ -1,0 +1,145 @@
+/*
+ * regtopk.h: C ABI of the RegTop-k sparsification step for N workers batched on one GPU.
+ *
+ * The calls follow the paper's statement of the method (arXiv 2501.05633):
+ *   - Algorithm 2 ("RegTop-k sparsification at worker n"): accumulate a = eps + g, posterior
+ *     distortion Delta on the previous mask's support (Eq. (Delta_def)), score
+ *     |a| * tanh(|1 + Delta| / mu), top-k mask of the score, send the raw accumulator on the mask,
+ *     residual eps' = a - ghat.  Round 0, and mu == 0, are Algorithm 1 (Top-k with error
+ *     accumulation).
+ *   - Section 2.2: the top-k selector and the server aggregation g = sum_n omega_n * ghat_n.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".
+ *   - The caller owns every buffer it passes, including the workspace; the library allocates no
+ *     device memory.  It owns only a small host-side context (malloc'ed by regtopk_create, freed by
+ *     regtopk_destroy).
+ *   - Calls enqueue work on the CUDA stream given at creation and return without synchronising,
+ *     except where stated.  Buffers must stay valid until that work has run.
+ *   - Return value: REGTOPK_OK (0) or a negative REGTOPK_ERR_* code.  Nothing aborts, throws or traps.
+ *   - Arithmetic: binary32, every operation individually rounded in the written order (no fused
+ *     multiply-add), so results are reproducible bit for bit; selection is exact, ties between equal
+ *     scores go to the lower index.  Gradients must be finite.
+ *   - One GPU, one context per (d, N, k) problem; contexts are independent.  A context is not
+ *     thread-safe.
+ */
+#ifndef REGTOPK_H_
+#define REGTOPK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct regtopk_ctx regtopk_ctx;
+
+enum {
+  REGTOPK_OK = 0,
+  REGTOPK_ERR_INVALID_ARG = -1,         /* a size, pointer, alignment or hyper-parameter is unusable   */
+  REGTOPK_ERR_WORKSPACE_TOO_SMALL = -2, /* workspace_bytes < regtopk_workspace_bytes(...)              */
+  REGTOPK_ERR_SEQUENCE = -3,            /* worker_step twice without aggregate, or aggregate first     */
+  REGTOPK_ERR_CUDA = -4,                /* a CUDA runtime call or launch failed                        */
+  REGTOPK_ERR_INTERNAL = -5,            /* the device reported an inconsistent selection (a bug)       */
+  REGTOPK_ERR_NO_DEVICE = -6            /* no usable sm_100 device / kernel image                      */
+};
+
+enum { REGTOPK_GRAD_F32 = 0, REGTOPK_GRAD_BF16 = 1 };
+
+/* flags of regtopk_params */
+enum {
+  REGTOPK_FLAG_HOST_STAGING = 1,      /* reserve workspace for regtopk_round_host                          */
+  REGTOPK_FLAG_FORCE_DENSE_SELECT = 2 /* testing: skip the sampled cutoff, always take the dense exact path */
+};
+
+typedef struct {
+  float mu;            /* > 0: RegTop-k (Algorithm 2).  == 0: Top-k with error accumulation (Algorithm 1). */
+  const float* omega;  /* host array of N aggregation weights (Eq. (1)), or NULL for 1/N each.             */
+  int32_t grad_dtype;  /* REGTOPK_GRAD_F32 or REGTOPK_GRAD_BF16; accumulators and residuals are binary32.  */
+  int32_t flags;       /* REGTOPK_FLAG_*                                                                   */
+} regtopk_params;
+
+/* Bytes of device workspace a context for (d, N, k) needs; 0 if the arguments are invalid.
+ * d = model size J, N = number of workers, k = entries kept per worker; 1 <= k <= d <= 2^31 - 2. */
+size_t regtopk_workspace_bytes(int64_t d, int32_t N, int64_t k, const regtopk_params* params);
+
+/* Algorithm 2, "Initialization": eps_n = 0 for every worker, no previous mask, round 0.
+ * workspace: device memory, 256-byte aligned, at least regtopk_workspace_bytes(...) bytes; the library
+ * keeps all state in it (residuals [N][ld] binary32, previous aggregate g [d], previous pairs, masks,
+ * candidate lists).  cuda_stream: a cudaStream_t (NULL = default stream).  *out receives the context
+ * (host).  Enqueues the clearing of the workspace.  Errors: INVALID_ARG, WORKSPACE_TOO_SMALL, CUDA,
+ * NO_DEVICE. */
+int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const regtopk_params* params,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* One sparsification round of all N workers: Algorithm 2 steps 6-12 (Algorithm 1 steps 2-7 in round 0
+ * or when mu == 0).
+ *   grads    [N][grad_ld] gradients g_n^t in the context's grad_dtype, row n at grads + n*grad_ld
+ *            elements; read-only.  grad_ld >= d.  Rows that are 16-byte aligned (fp32: grad_ld % 4 == 0
+ *            and an aligned base; bf16: 8-byte, grad_ld % 4 == 0) take the vectorised path; any other
+ *            layout is accepted and read element by element.
+ *   out_idx  [N][k] int32: worker n's mask support in ascending order.
+ *   out_val  [N][k] binary32: the accumulator a_n^t at those indices (not the score).
+ * Exactly k pairs per worker are written.  Afterwards the residual state holds eps^{t+1}.
+ * Errors: INVALID_ARG (NULL pointer, grad_ld < d), SEQUENCE (previous round not aggregated), CUDA. */
+int regtopk_worker_step(regtopk_ctx* ctx, const void* grads, int64_t grad_ld, int32_t* out_idx,
+                        float* out_val);
+
+/* Server side of the round (Section 2.2): g^t = sum_n omega_n * ghat_n^t, workers added in the order
+ * n = 0..N-1 with each product rounded before its addition, then the state roll for round t+1 (the
+ * pairs just sent become the previous mask and a^{t} on it, g^t becomes g^{t-1}).
+ *   out_g    [d] binary32 or NULL; if given, receives a copy of g^t.
+ * Errors: SEQUENCE (no worker_step since the last aggregate), CUDA. */
+int regtopk_aggregate(regtopk_ctx* ctx, float* out_g);
+
+/* Device pointer to the library's own copy of the latest aggregate g^t ([d] binary32, inside the
+ * workspace, valid until the next regtopk_aggregate is enqueued).  *dev_ptr is written on the host. */
+int regtopk_global_gradient(regtopk_ctx* ctx, const float** dev_ptr);
+
+/* Back to Algorithm 2's initial state: eps = 0, no previous mask, g = 0, round 0. */
+int regtopk_state_reset(regtopk_ctx* ctx);
+
+/* One whole round from HOST buffers: copies h_grads ([N][grad_ld], pinned memory recommended) to the
+ * device staging area, runs regtopk_worker_step and regtopk_aggregate, copies the pairs (and g if
+ * h_g != NULL) back to host memory, and SYNCHRONISES the stream before returning.  Needs
+ * REGTOPK_FLAG_HOST_STAGING at creation and grad_ld <= d rounded up to a multiple of 1024 (the row
+ * length reserved for staging).  h_idx [N][k], h_val [N][k], h_g [d] or NULL: host. */
+int regtopk_round_host(regtopk_ctx* ctx, const void* h_grads, int64_t grad_ld, int32_t* h_idx,
+                       float* h_val, float* h_g);
+
+/* Synchronises the stream and returns REGTOPK_OK or the sticky error recorded by the device
+ * (REGTOPK_ERR_INTERNAL) or by CUDA (REGTOPK_ERR_CUDA). */
+int regtopk_status(regtopk_ctx* ctx);
+
+typedef struct {
+  int64_t rounds;               /* worker_step calls so far                                               */
+  int64_t kernel_launches;      /* kernels launched by this context so far                                */
+  int64_t dense_select_workers; /* worker-rounds that needed the dense exact path (sampled cutoff missed) */
+  int64_t candidates_last;      /* candidates gathered in the last round, summed over workers             */
+  int64_t candidate_capacity;   /* per-worker capacity of the candidate list                              */
+} regtopk_stats;
+
+/* Synchronises the stream and fills *out (host). */
+int regtopk_get_stats(regtopk_ctx* ctx, regtopk_stats* out);
+
+/* Per-kernel timing with CUDA events on the context's stream.  enable != 0 starts recording an event
+ * pair around the streaming accumulate kernel of every following worker_step (up to 4096 calls);
+ * regtopk_profile_read synchronises and returns the summed milliseconds and the number of calls, then
+ * clears the record.  Both outputs are host pointers. */
+int regtopk_profile_enable(regtopk_ctx* ctx, int enable);
+int regtopk_profile_read(regtopk_ctx* ctx, double* stream_kernel_ms, int64_t* calls);
+
+/* Test introspection: device pointer to the residuals eps ([N][*ld] binary32, *ld >= d). */
+int regtopk_debug_residual(regtopk_ctx* ctx, const float** dev_ptr, int64_t* ld);
+
+/* Frees the host-side context.  Synchronises the stream first.  The workspace is the caller's. */
+int regtopk_destroy(regtopk_ctx* ctx);
+
+/* Static, human-readable text for a return code. */
+const char* regtopk_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REGTOPK_H_ */

@@ -1,0 +1,251 @@
+"""Thin ctypes binding of include/regtopk.h: argument marshalling only.
+
+torch is used for device memory and streams; every step of the method runs in libregtopk.so.
+There is no CPU path: if the library is missing or no CUDA device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_ROOT = os.path.dirname(_PKG)
+_SRC = os.path.join(_PKG, "csrc", "regtopk.cu")
+_INC = os.path.join(_ROOT, "include")
+_LIB = os.path.join(_PKG, "libregtopk.so")
+
+OK = 0
+GRAD_F32, GRAD_BF16 = 0, 1
+FLAG_HOST_STAGING, FLAG_FORCE_DENSE_SELECT = 1, 2
+
+EXPORTS = [
+    "regtopk_workspace_bytes", "regtopk_create", "regtopk_worker_step", "regtopk_aggregate",
+    "regtopk_global_gradient", "regtopk_state_reset", "regtopk_round_host", "regtopk_status",
+    "regtopk_get_stats", "regtopk_profile_enable", "regtopk_profile_read", "regtopk_debug_residual",
+    "regtopk_destroy", "regtopk_strerror",
+]
+
+
+class Params(ctypes.Structure):
+    _fields_ = [("mu", ctypes.c_float), ("omega", ctypes.POINTER(ctypes.c_float)),
+                ("grad_dtype", ctypes.c_int32), ("flags", ctypes.c_int32)]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [("rounds", ctypes.c_int64), ("kernel_launches", ctypes.c_int64),
+                ("dense_select_workers", ctypes.c_int64), ("candidates_last", ctypes.c_int64),
+                ("candidate_capacity", ctypes.c_int64)]
+
+
+def library_path() -> str:
+    return _LIB
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile csrc/regtopk.cu for sm_100a into the package directory (nvcc cross-compiles without a GPU)."""
+    if not force and os.path.exists(_LIB) and os.path.getmtime(_LIB) >= max(
+            os.path.getmtime(_SRC), os.path.getmtime(os.path.join(_INC, "regtopk.h"))):
+        return _LIB
+    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "-I", _INC, "--shared", "-Xcompiler", "-fPIC", "-o", _LIB, _SRC]
+    if verbose:
+        cmd.insert(1, "-Xptxas=-v")
+    subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+
+
+def load_library():
+    """dlopen the CUDA library and declare its signatures. Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB):
+        raise RuntimeError(f"{_LIB} is missing: run paper_2501_05633_b200.build() (needs nvcc); "
+                           "there is no CPU implementation to fall back to")
+    L = ctypes.CDLL(_LIB)
+    vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
+    L.regtopk_workspace_bytes.restype = ctypes.c_size_t
+    L.regtopk_workspace_bytes.argtypes = [i64, i32, i64, ctypes.POINTER(Params)]
+    L.regtopk_create.restype = ctypes.c_int
+    L.regtopk_create.argtypes = [ctypes.POINTER(vp), i64, i32, i64, ctypes.POINTER(Params), vp,
+                                 ctypes.c_size_t, vp]
+    L.regtopk_worker_step.restype = ctypes.c_int
+    L.regtopk_worker_step.argtypes = [vp, vp, i64, vp, vp]
+    L.regtopk_aggregate.restype = ctypes.c_int
+    L.regtopk_aggregate.argtypes = [vp, vp]
+    L.regtopk_global_gradient.restype = ctypes.c_int
+    L.regtopk_global_gradient.argtypes = [vp, ctypes.POINTER(vp)]
+    L.regtopk_state_reset.restype = ctypes.c_int
+    L.regtopk_state_reset.argtypes = [vp]
+    L.regtopk_round_host.restype = ctypes.c_int
+    L.regtopk_round_host.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.regtopk_status.restype = ctypes.c_int
+    L.regtopk_status.argtypes = [vp]
+    L.regtopk_get_stats.restype = ctypes.c_int
+    L.regtopk_get_stats.argtypes = [vp, ctypes.POINTER(Stats)]
+    L.regtopk_profile_enable.restype = ctypes.c_int
+    L.regtopk_profile_enable.argtypes = [vp, ctypes.c_int]
+    L.regtopk_profile_read.restype = ctypes.c_int
+    L.regtopk_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
+    L.regtopk_debug_residual.restype = ctypes.c_int
+    L.regtopk_debug_residual.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i64)]
+    L.regtopk_destroy.restype = ctypes.c_int
+    L.regtopk_destroy.argtypes = [vp]
+    L.regtopk_strerror.restype = ctypes.c_char_p
+    L.regtopk_strerror.argtypes = [ctypes.c_int]
+    _lib = L
+    return L
+
+
+class RegTopKError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = load_library().regtopk_strerror(code).decode()
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise RegTopKError(code, where)
+
+
+def _make_params(mu, omega, grad_dtype, flags):
+    p = Params()
+    p.mu = float(mu)
+    keep = None
+    if omega is not None:
+        keep = (ctypes.c_float * len(omega))(*[float(x) for x in omega])
+        p.omega = ctypes.cast(keep, ctypes.POINTER(ctypes.c_float))
+    p.grad_dtype = grad_dtype
+    p.flags = flags
+    return p, keep
+
+
+def workspace_bytes(d, N, k, mu=4.0, omega=None, grad_dtype=GRAD_F32, flags=0) -> int:
+    p, _keep = _make_params(mu, omega, grad_dtype, flags)
+    return int(load_library().regtopk_workspace_bytes(d, N, k, ctypes.byref(p)))
+
+
+class RegTopK:
+    """One (d, N, k) sparsifier context on the current CUDA device.
+
+    grads: torch tensor [N, ld] on the device, float32 or bfloat16 as chosen at construction.
+    worker_step returns (idx [N,k] int32, val [N,k] float32); aggregate returns g [d] float32 (a view of
+    the library's state unless `out` is given).  Work is enqueued on `stream` (default: torch's current
+    stream at construction) and is asynchronous like any torch CUDA op.
+    """
+
+    def __init__(self, d: int, N: int, k: int, mu: float = 4.0, omega=None, grad_dtype=torch.float32,
+                 flags: int = 0, device=None, stream: Optional[torch.cuda.Stream] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("RegTopK needs a CUDA device; there is no CPU implementation")
+        self.L = load_library()
+        self.device = torch.device(device if device is not None else f"cuda:{torch.cuda.current_device()}")
+        self.d, self.N, self.k, self.mu = int(d), int(N), int(k), float(mu)
+        self.torch_dtype = grad_dtype
+        self.dtype_code = GRAD_BF16 if grad_dtype == torch.bfloat16 else GRAD_F32
+        if grad_dtype not in (torch.float32, torch.bfloat16):
+            raise TypeError("gradients are float32 or bfloat16")
+        self.flags = int(flags)
+        p, keep = _make_params(mu, omega, self.dtype_code, self.flags)
+        nbytes = int(self.L.regtopk_workspace_bytes(self.d, self.N, self.k, ctypes.byref(p)))
+        if nbytes == 0:
+            raise RegTopKError(-1, "regtopk_workspace_bytes")
+        with torch.cuda.device(self.device):
+            self.stream = stream if stream is not None else torch.cuda.current_stream()
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            ctx = ctypes.c_void_p()
+            _check(self.L.regtopk_create(ctypes.byref(ctx), self.d, self.N, self.k, ctypes.byref(p),
+                                         self.workspace.data_ptr(), nbytes, self.stream.cuda_stream),
+                   "regtopk_create")
+        self.ctx = ctx
+        self.workspace_nbytes = nbytes
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            self.L.regtopk_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check_grads(self, grads: torch.Tensor):
+        if grads.dtype != self.torch_dtype or grads.dim() != 2 or grads.shape[0] != self.N:
+            raise TypeError("grads must be [N, ld] of the context's dtype")
+        if grads.shape[1] < self.d or grads.stride(1) != 1:
+            raise ValueError("grads rows must be contiguous with ld >= d")
+        return int(grads.stride(0)) if self.N > 1 else int(grads.shape[1])
+
+    def worker_step(self, grads: torch.Tensor, out_idx: Optional[torch.Tensor] = None,
+                    out_val: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+        if not grads.is_cuda:
+            raise TypeError("grads must live on the device (use round_host for host buffers)")
+        ld = self._check_grads(grads)
+        if out_idx is None:
+            out_idx = torch.empty((self.N, self.k), dtype=torch.int32, device=self.device)
+        if out_val is None:
+            out_val = torch.empty((self.N, self.k), dtype=torch.float32, device=self.device)
+        _check(self.L.regtopk_worker_step(self.ctx, grads.data_ptr(), ld, out_idx.data_ptr(),
+                                          out_val.data_ptr()), "regtopk_worker_step")
+        return out_idx, out_val
+
+    def aggregate(self, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        _check(self.L.regtopk_aggregate(self.ctx, out.data_ptr() if out is not None else None),
+               "regtopk_aggregate")
+        return out if out is not None else self.global_gradient()
+
+    def global_gradient(self) -> torch.Tensor:
+        """View of the library's g^t inside the workspace (overwritten by the next aggregate)."""
+        ptr = ctypes.c_void_p()
+        _check(self.L.regtopk_global_gradient(self.ctx, ctypes.byref(ptr)), "regtopk_global_gradient")
+        off = ptr.value - self.workspace.data_ptr()
+        return self.workspace[off: off + 4 * self.d].view(torch.float32)
+
+    def residual(self) -> torch.Tensor:
+        """View [N, d] of the residuals eps (test introspection)."""
+        ptr, ld = ctypes.c_void_p(), ctypes.c_int64()
+        _check(self.L.regtopk_debug_residual(self.ctx, ctypes.byref(ptr), ctypes.byref(ld)),
+               "regtopk_debug_residual")
+        off = ptr.value - self.workspace.data_ptr()
+        full = self.workspace[off: off + 4 * self.N * ld.value].view(torch.float32).view(self.N, ld.value)
+        return full[:, : self.d]
+
+    def state_reset(self):
+        _check(self.L.regtopk_state_reset(self.ctx), "regtopk_state_reset")
+
+    def round_host(self, h_grads: torch.Tensor, h_idx: torch.Tensor, h_val: torch.Tensor,
+                   h_g: Optional[torch.Tensor] = None):
+        """A whole round from host tensors (pinned recommended); synchronises before returning."""
+        if h_grads.is_cuda or h_idx.is_cuda or h_val.is_cuda:
+            raise TypeError("round_host takes host tensors")
+        ld = self._check_grads(h_grads)
+        _check(self.L.regtopk_round_host(self.ctx, h_grads.data_ptr(), ld, h_idx.data_ptr(),
+                                         h_val.data_ptr(), h_g.data_ptr() if h_g is not None else None),
+               "regtopk_round_host")
+
+    def status(self):
+        _check(self.L.regtopk_status(self.ctx), "regtopk_status")
+
+    def stats(self) -> dict:
+        s = Stats()
+        _check(self.L.regtopk_get_stats(self.ctx, ctypes.byref(s)), "regtopk_get_stats")
+        return {n: int(getattr(s, n)) for n, _ in Stats._fields_}
+
+    def profile_enable(self, enable: bool = True):
+        _check(self.L.regtopk_profile_enable(self.ctx, 1 if enable else 0), "regtopk_profile_enable")
+
+    def profile_read(self) -> Tuple[float, int]:
+        ms, calls = ctypes.c_double(), ctypes.c_int64()
+        _check(self.L.regtopk_profile_read(self.ctx, ctypes.byref(ms), ctypes.byref(calls)),
+               "regtopk_profile_read")
+        return float(ms.value), int(calls.value)

@@ -1,0 +1,292 @@
+"""CUDA library against the CPU oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2501_05633_b200 import RegTopK, binding, synth
+from paper_2501_05633_b200.binding import RegTopKError
+from tests.parity import run_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def gauss_rounds(N, d, T, seed, ld=None, scale=None, dtype=torch.float32, quant=None):
+    g = torch.Generator().manual_seed(seed)
+    ld = ld or d
+    for t in range(T):
+        x = torch.zeros((N, ld), dtype=torch.float32)
+        v = torch.randn((N, d), generator=g)
+        if scale is not None:
+            v = v * scale
+        if quant:
+            v = torch.round(v * quant) / quant
+        x[:, :d] = v
+        yield x.to(dtype)
+
+
+# ---- tiny and ragged sizes, every k regime -----------------------------------------------------------
+@pytest.mark.parametrize("d,N,k", [(1, 1, 1), (2, 2, 1), (7, 3, 7), (33, 2, 5), (511, 2, 17), (512, 1, 512),
+                                   (513, 3, 1), (4096, 8, 41), (65536, 2, 100), (65537, 2, 655),
+                                   (200003, 4, 2000), (200003, 2, 200003), (1_000_003, 2, 1000)])
+@pytest.mark.parametrize("mu", [4.0, 0.0])
+def test_sizes(d, N, k, mu):
+    run_parity(gauss_rounds(N, d, 4, seed=d + N), d, N, k, mu)
+
+
+@pytest.mark.parametrize("mu", [1.0, 4.0, 10.0, 1e-30])
+def test_mu_sweep(mu):
+    run_parity(gauss_rounds(4, 50_001, 5, seed=3), 50_001, 4, 500, mu)
+
+
+def test_custom_weights():
+    run_parity(gauss_rounds(3, 30_000, 4, seed=5), 30_000, 3, 300, 4.0, omega=[0.3, 0.5, 0.2])
+
+
+@pytest.mark.parametrize("ld_extra", [0, 1, 2, 3, 5])
+def test_unaligned_rows(ld_extra):
+    d = 100_001
+    run_parity(gauss_rounds(3, d, 3, seed=9, ld=d + ld_extra), d, 3, 1000, 4.0)
+
+
+def test_unaligned_base_pointer():
+    d, N, k = 40_000, 2, 400
+    rounds = []
+    for x in gauss_rounds(N, d, 3, seed=4, ld=d + 4):
+        buf = torch.zeros(N * (d + 4) + 1)
+        view = buf[1:].view(N, d + 4)  # base pointer 4 bytes off a 16-byte boundary
+        view.copy_(x)
+        rounds.append(view)
+
+    class DevRounds:
+        def __iter__(self):
+            for v in rounds:
+                dbuf = torch.zeros(N * (d + 4) + 1, device="cuda")
+                dv = dbuf[1:].view(N, d + 4)
+                dv.copy_(v)
+                yield dv
+
+    run_parity(DevRounds(), d, N, k, 4.0)
+
+
+# ---- degenerate inputs ---------------------------------------------------------------------------------
+def test_all_zero_gradients():
+    d, N, k = 70_001, 2, 700
+    run_parity([torch.zeros(N, d) for _ in range(3)], d, N, k, 4.0, expect_dense=True)
+
+
+def test_all_equal_gradients():
+    d, N, k = 70_001, 2, 700
+    run_parity([torch.full((N, d), 0.5), torch.full((N, d), -0.25), torch.full((N, d), 0.5)], d, N, k, 4.0,
+               expect_dense=True)
+
+
+def test_fewer_nonzeros_than_k():
+    d, N, k = 100_000, 3, 1000
+    rounds = []
+    g = torch.Generator().manual_seed(1)
+    for t in range(4):
+        x = torch.zeros(N, d)
+        pos = torch.randint(0, d, (N, 300), generator=g)
+        x.scatter_(1, pos, torch.randn(N, 300, generator=g))
+        rounds.append(x)
+    run_parity(rounds, d, N, k, 4.0)
+
+
+def test_heavy_ties():
+    run_parity(gauss_rounds(3, 150_000, 5, seed=8, quant=2), 150_000, 3, 1500, 4.0)
+    run_parity(gauss_rounds(3, 150_000, 4, seed=8, quant=2), 150_000, 3, 1500, 4.0,
+               flags=binding.FLAG_FORCE_DENSE_SELECT)
+
+
+def test_bf16_gradients():
+    run_parity(gauss_rounds(4, 120_007, 5, seed=12, ld=120_008, dtype=torch.bfloat16), 120_007, 4, 1200, 4.0)
+    run_parity(gauss_rounds(2, 120_007, 3, seed=13, ld=120_007, dtype=torch.bfloat16), 120_007, 2, 120, 4.0)
+
+
+def test_denormals_and_huge_values():
+    d, N = 60_000, 2
+    g = torch.Generator().manual_seed(2)
+    rounds = []
+    for t in range(4):
+        x = torch.randn(N, d, generator=g)
+        x[:, ::3] *= 1e-42  # subnormal accumulators
+        x[:, 1::7] *= 1e30
+        rounds.append(x)
+    run_parity(rounds, d, N, 600, 4.0)
+
+
+# ---- the dense exact path --------------------------------------------------------------------------------
+@pytest.mark.parametrize("mu", [4.0, 0.0])
+def test_forced_dense_select(mu):
+    run_parity(gauss_rounds(3, 90_001, 5, seed=21), 90_001, 3, 900, mu, flags=binding.FLAG_FORCE_DENSE_SELECT,
+               expect_dense=True)
+
+
+def _sample_positions(d):
+    Q = (d + 7) // 8
+    s = np.arange(4096, dtype=np.int64)
+    q = s * Q // 4096
+    return (q[:, None] * 8 + np.arange(8)[None, :]).reshape(-1)
+
+
+def test_sample_overestimates_cutoff():
+    """Large entries sit exactly where the cutoff sample looks: the guess is too high, too few
+    candidates are gathered, and the dense path must still give the exact mask."""
+    d, N, k = 1_000_000, 2, 5000
+    pos = torch.from_numpy(_sample_positions(d))
+    rounds = []
+    for x in gauss_rounds(N, d, 3, seed=30):
+        x[:, pos] *= 100.0
+        rounds.append(x)
+    run_parity(rounds, d, N, k, 4.0, expect_dense=True)
+
+
+def test_sample_underestimates_cutoff():
+    """Large entries sit only where the sample does not look: the guess is too low and the candidate
+    list overflows."""
+    d, N, k = 1_000_000, 2, 200
+    keep = torch.ones(d, dtype=torch.bool)
+    keep[torch.from_numpy(_sample_positions(d))] = False
+    rounds = []
+    for x in gauss_rounds(N, d, 3, seed=31):
+        x[:, ~keep] *= 1e-3
+        rounds.append(x)
+    run_parity(rounds, d, N, k, 4.0, expect_dense=True)
+
+
+# ---- model-shaped workloads, scaled down (several tiles, ragged tail) ---------------------------------
+@pytest.mark.parametrize("name", ["resnet18", "resnet50", "gpt2", "flat1p3b"])
+def test_scaled_workloads(name):
+    w = synth.workload(name, scale_to=300_000)
+    stream = synth.GradientStream(w, device="cpu", seed=17, pad_to=8)
+    for k in w.k_values():
+        k = max(k, 1)
+        s = synth.GradientStream(w, device="cpu", seed=17, pad_to=8)
+        run_parity((s.next() for _ in range(6)), w.d, w.N, k, w.mu)
+
+
+def test_least_squares_trajectory():
+    """N=8, 512x4096 least squares, k=41, 100 rounds with step 0.1: identical masks, residuals and
+    aggregates every round, hence the identical loss curve, which must fall."""
+    from oracle.oracle import OracleRegTopK
+    prob = synth.LeastSquares()
+    lib = RegTopK(prob.d, prob.N, 41, mu=4.0)
+    ora = OracleRegTopK(prob.d, prob.N, 41, 4.0)
+    th_l = np.zeros(prob.d)
+    th_o = np.zeros(prob.d)
+    losses = [prob.loss(th_l)]
+    for t in range(100):
+        g_l = prob.gradients(th_l)
+        g_o = prob.gradients(th_o)
+        idx, val = lib.worker_step(torch.from_numpy(g_l).cuda())
+        oi, ov = ora.worker_step(g_o)
+        assert np.array_equal(idx.cpu().numpy(), oi) and np.array_equal(val.cpu().numpy().view(np.uint32), ov.view(np.uint32))
+        assert np.array_equal(lib.residual().cpu().numpy().view(np.uint32), ora.eps.view(np.uint32))
+        agg = lib.aggregate().cpu().numpy()
+        assert np.array_equal(agg.view(np.uint32), ora.aggregate().view(np.uint32))
+        th_l = th_l - 0.1 * agg.astype(np.float64)
+        th_o = th_l.copy()
+        losses.append(prob.loss(th_l))
+    lib.status()
+    assert losses[-1] < 0.9 * losses[0]
+    assert losses[50] < losses[0]
+
+
+# ---- API behaviour -------------------------------------------------------------------------------------------
+def test_state_reset_restarts_at_round_zero():
+    run_parity(gauss_rounds(2, 20_000, 6, seed=40), 20_000, 2, 200, 4.0, reset_after=3)
+
+
+def test_sequence_errors():
+    lib = RegTopK(1000, 2, 10)
+    g = torch.randn(2, 1000, device="cuda")
+    with pytest.raises(RegTopKError) as e:
+        lib.aggregate()
+    assert e.value.code == -3
+    lib.worker_step(g)
+    with pytest.raises(RegTopKError) as e:
+        lib.worker_step(g)
+    assert e.value.code == -3
+    lib.aggregate()
+    lib.worker_step(g)
+    lib.aggregate()
+    lib.status()
+
+
+def test_argument_errors():
+    lib = RegTopK(1000, 2, 10)
+    L = lib.L
+    g = torch.randn(2, 1000, device="cuda")
+    oi = torch.empty(2, 10, dtype=torch.int32, device="cuda")
+    ov = torch.empty(2, 10, device="cuda")
+    assert L.regtopk_worker_step(lib.ctx, g.data_ptr(), 999, oi.data_ptr(), ov.data_ptr()) == -1
+    assert L.regtopk_worker_step(lib.ctx, None, 1000, oi.data_ptr(), ov.data_ptr()) == -1
+    assert L.regtopk_worker_step(lib.ctx, g.data_ptr(), 1000, None, ov.data_ptr()) == -1
+    hi = torch.empty(2, 10, dtype=torch.int32)
+    hv = torch.empty(2, 10)
+    with pytest.raises(RegTopKError):  # no staging reserved
+        lib.round_host(g.cpu(), hi, hv)
+    import ctypes
+    ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    p, _ = binding._make_params(4.0, None, 0, 0)
+    ctx = ctypes.c_void_p()
+    assert L.regtopk_create(ctypes.byref(ctx), 1000, 2, 10, ctypes.byref(p), ws.data_ptr(), 1024, None) == -2
+    assert L.regtopk_create(ctypes.byref(ctx), 1000, 2, 10, ctypes.byref(p), ws.data_ptr() + 4, 10**9, None) == -1
+
+
+def test_determinism_and_output_copy():
+    d, N, k = 300_000, 4, 3000
+    rounds = [x.cuda() for x in gauss_rounds(N, d, 4, seed=50)]
+    outs = []
+    for rep in range(2):
+        lib = RegTopK(d, N, k)
+        rec = []
+        for g in rounds:
+            idx, val = lib.worker_step(g)
+            og = torch.empty(d, device="cuda")
+            ret = lib.aggregate(out=og)
+            assert ret is og and torch.equal(og, lib.global_gradient())
+            rec.append((idx.clone(), val.clone(), og.clone(), lib.residual().clone()))
+        lib.status()
+        outs.append(rec)
+    for a, b in zip(*outs):
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+
+
+def test_round_host_matches_device_calls():
+    d, N, k = 120_000, 3, 1200
+    rounds = list(gauss_rounds(N, d, 4, seed=60))
+    dev = RegTopK(d, N, k)
+    host = RegTopK(d, N, k, flags=binding.FLAG_HOST_STAGING)
+    for g in rounds:
+        idx, val = dev.worker_step(g.cuda())
+        agg = dev.aggregate()
+        hi = torch.empty(N, k, dtype=torch.int32).pin_memory()
+        hv = torch.empty(N, k).pin_memory()
+        hg = torch.empty(d).pin_memory()
+        host.round_host(g.pin_memory(), hi, hv, hg)
+        assert torch.equal(hi, idx.cpu()) and torch.equal(hv, val.cpu()) and torch.equal(hg, agg.cpu())
+    host.status()
+
+
+def test_fast_path_is_taken_on_ordinary_data():
+    w = synth.workload("resnet18", scale_to=2_000_000)
+    s = synth.GradientStream(w, device="cuda", seed=3, pad_to=8)
+    lib = RegTopK(w.d, w.N, w.k_values()[0])
+    for t in range(6):
+        lib.worker_step(s.next())
+        lib.aggregate()
+    lib.status()
+    st = lib.stats()
+    assert st["dense_select_workers"] == 0, st
+    assert st["candidates_last"] <= w.N * st["candidate_capacity"]
+
+
+# ---- full benchmark sizes, in the layout the benchmark times -------------------------------------------------
+@pytest.mark.parametrize("name,ki,rounds", [("resnet18", 0, 3), ("resnet18", 1, 2), ("resnet50", 0, 2)])
+def test_full_size_workloads(name, ki, rounds):
+    w = synth.workload(name)
+    s = synth.GradientStream(w, device="cuda", seed=0, pad_to=32)
+    run_parity((s.next() for _ in range(rounds)), w.d, w.N, w.k_values()[ki], w.mu, select_mode=1, threads=8,
+               expect_dense=False)
