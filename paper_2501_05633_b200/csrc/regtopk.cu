@@ -1,20 +1,21 @@
 // RegTop-k sparsification step for N workers batched on one B200 (sm_100a): kernels and C ABI.
 //
-// One round (regtopk_worker_step + regtopk_aggregate) is this chain of kernels on one stream:
+// One round (regtopk_worker_step + regtopk_aggregate) is four kernels on one stream:
 //
-//   k_sample_cutoff   per worker: read a strided sample of a = eps + g, pick a candidate cutoff key
-//                     from the sample's order statistics (a guess that only has to be low enough)
-//   k_stream          the one Theta(N*d) pass: a = eps + g written in place over eps, every entry
-//                     whose key bits(|a|) reaches the cutoff appended to the worker's candidate list
-//   k_override        the <= k entries of the previous mask's support: posterior distortion,
-//                     tanh regulariser, regularised score (Algorithm 2 steps 8-9)
-//   k_select          per worker: exact radix select of the k largest (score, lowest index) among
-//                     candidates + overrides; winners are set in a bitmask
-//   k_dense_select    only for a worker whose cutoff guess was too high or whose list overflowed:
-//                     exact radix select over the whole row (slow, always right)
-//   k_select (again)  takes over the winners of the dense path
-//   k_emit            ordered walk of the bitmask: ascending (index, a[index]) pairs, residual zeroed
-//   k_aggregate       server sum in worker order, clearing last round's entries first
+//   k_sample_cutoff   one block per worker: reads a strided sample of a = eps + g and derives, from
+//                     the sample's order statistics, a candidate cutoff key (a guess that only has to
+//                     be low enough) and the bin width the select will use
+//   k_stream          the one Theta(N*d) pass: a = eps + g written in place over eps; every entry
+//                     whose key bits(|a|) reaches the cutoff is appended to the worker's candidate list
+//   k_post            one thread-block cluster per worker (distributed shared memory for the
+//                     histogram merge): regularised scores on the previous mask's support
+//                     (Eq. (Delta_def), Algorithm 2 steps 8-9), exact selection of the k largest
+//                     (score, lowest index) among candidates and overrides, winners set in a bitmask,
+//                     ordered walk of the bitmask emitting ascending (index, a[index]) pairs and
+//                     zeroing the residual there.  If the cutoff guess was too high or the list
+//                     overflowed, the same cluster runs an exact radix select over the whole row.
+//   k_aggregate       server sum in worker order, one thread per sent pair, ranks looked up through
+//                     the per-word prefix counts written during emission
 //
 // The selection key of an entry is the bit pattern of its non-negative binary32 score, which orders
 // like the score; the 64-bit composite (key << 32 | ~index) orders like (score descending, index
@@ -25,38 +26,45 @@
 // ever written: the accumulator that has to be stored anyway is the only dense output.
 //
 // All floating-point steps use the round-to-nearest intrinsics, which the compiler never contracts
-// into fused multiply-adds.
+// into fused multiply-adds.  No kernel waits on another block except through the hardware cluster
+// barrier, which every block of a cluster reaches the same number of times.
 
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
+#include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
-#include <math.h>
 
 #include "regtopk.h"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
 typedef unsigned long long u64;
 typedef uint32_t u32;
 
-constexpr int kTileWords = 2048;           // bitmask words per emission tile
-constexpr int kTileShift = 16;             // log2(coordinates per tile) = log2(2048 * 32)
 constexpr int kSampleSectors = 4096;       // 32-byte sectors sampled per worker
 constexpr int kSampleMax = kSampleSectors * 8;
 constexpr int kBlockSel = 1024;            // threads of the per-worker kernels
 constexpr int kStreamThreads = 256;
 constexpr int kWarpList = 256;             // per-warp staging list of k_stream (entries)
+constexpr int kBins = 4096;                // histogram bins of the select
+constexpr int kMaxCluster = 16;
 constexpr u32 kFull = 0xFFFFFFFFu;
 
-enum : u32 { kStateNormal = 0, kStateNeedDense = 1, kStateDenseDone = 2 };
-enum : u32 { kErrCountMismatch = 1u, kErrDenseSelect = 2u };
+enum : u32 { kErrCountMismatch = 1u, kErrDenseSelect = 2u, kErrRefine = 4u };
 
 struct WorkerCtl {
-  u32 cutoff;      // candidate cutoff key of this round
-  u32 cand_count;  // entries appended (may exceed the capacity: then the list overflowed)
-  u32 state;       // kState*
-  u32 n_valid;     // valid items seen by the select (diagnostics)
+  u32 cutoff;       // candidate cutoff key of this round
+  u32 bin_shift;    // select bins: bin = min(kBins - 1, (key - cutoff) >> bin_shift)
+  u32 cand_count;   // entries appended by k_stream (may exceed the capacity: the list overflowed)
+  u32 force_dense;  // skip the candidate path (testing flag)
+  u32 bcount;       // length of the refinement list
+  u32 acount;       // dense path: entries above the threshold gathered so far
+  u32 n_valid;      // valid items seen by the select (diagnostics)
+  u32 pad;
 };
 
 struct GlobalCtl {
@@ -187,6 +195,7 @@ __device__ __forceinline__ float load_grad(const void* row, int64_t j) {
   }
 }
 
+
 // ---------------------------------------------------------------------------------------------
 // k_sample_cutoff: one block per worker.
 // ---------------------------------------------------------------------------------------------
@@ -196,11 +205,10 @@ struct SampleArgs {
   const float* eps;
   int64_t ld;
   int64_t d;
+  int64_t k;
   int64_t k_target;  // entries the cutoff should leave above it (k, or 2k when overrides can demote)
   WorkerCtl* ctl;
   GlobalCtl* gctl;
-  u32* tcount;
-  int ntiles;
   int force_dense;
 };
 
@@ -208,20 +216,22 @@ template <bool BF16>
 __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
   extern __shared__ u32 s_dyn[];
   u32* s_keys = s_dyn;               // kSampleMax
-  u32* s_hist = s_dyn + kSampleMax;  // 4096
+  u32* s_hist = s_dyn + kSampleMax;  // kBins
   __shared__ u32 s_scan[33];
   __shared__ u32 s_res[3];
   const int n = blockIdx.x;
   const int tid = threadIdx.x;
+  WorkerCtl* ctl = p.ctl + n;
 
-  for (int t = tid; t < p.ntiles; t += blockDim.x) p.tcount[(size_t)n * p.ntiles + t] = 0;
   if (p.force_dense) {
     if (tid == 0) {
-      p.ctl[n].cutoff = kFull;  // no key reaches it: the stream pass collects nothing
-      p.ctl[n].cand_count = 0;
-      p.ctl[n].state = kStateNeedDense;
-      p.ctl[n].n_valid = 0;
-      atomicAdd(&p.gctl->dense_workers, 1ull);
+      ctl->cutoff = kFull;  // no key reaches it: the stream pass collects nothing
+      ctl->bin_shift = 0;
+      ctl->cand_count = 0;
+      ctl->force_dense = 1;
+      ctl->bcount = 0;
+      ctl->acount = 0;
+      ctl->n_valid = 0;
     }
     return;
   }
@@ -233,33 +243,55 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
   const float* eps_row = p.eps + (size_t)n * p.ld;
   const char* grow = static_cast<const char*>(p.grads) + (size_t)n * p.grad_ld * (BF16 ? 2 : 4);
 
-  for (int i = tid; i < 4096; i += blockDim.x) s_hist[i] = 0;
+  for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
   __syncthreads();
-  for (int i = tid; i < nsect * 8; i += blockDim.x) {
-    const int s = i >> 3, e = i & 7;
-    const int64_t q = all ? s : (int64_t)(((u64)s * (u64)Q) / (u64)kSampleSectors);
-    const int64_t j = q * 8 + e;
-    u32 key = 0;
-    if (j < p.d) {
-      const float a = __fadd_rn(eps_row[j], load_grad<BF16>(grow, j));
-      key = __float_as_uint(a) & 0x7FFFFFFFu;
-      atomicAdd(&s_hist[key >> 19], 1u);
+  // eight independent sample loads in flight per thread
+  for (int i0 = 0; i0 < nsect * 8; i0 += 8 * kBlockSel) {
+    float e[8], g[8];
+    bool ok[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * kBlockSel + tid;
+      const int s = i >> 3;
+      const int64_t q = all ? s : (int64_t)(((u64)s * (u64)Q) / (u64)kSampleSectors);
+      const int64_t j = q * 8 + (i & 7);
+      ok[u] = i < nsect * 8 && j < p.d;
+      e[u] = ok[u] ? eps_row[j] : 0.0f;
+      g[u] = ok[u] ? load_grad<BF16>(grow, j) : 0.0f;
     }
-    s_keys[i] = key;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * kBlockSel + tid;
+      u32 key = kFull;  // marks a slot outside the row
+      if (ok[u]) {
+        key = __float_as_uint(__fadd_rn(e[u], g[u])) & 0x7FFFFFFFu;
+        atomicAdd(&s_hist[key >> 19], 1u);
+      }
+      if (i < nsect * 8) s_keys[i] = key;
+    }
   }
   __syncthreads();
 
-  // rank to read off the sample: expected sample count above the target quantile plus a margin of
-  // four standard deviations (the count is close to Poisson) and a constant
-  u32 r;
-  {
-    const double lam = (double)p.k_target * (double)M / (double)p.d;
-    double rr = (M == p.d) ? (double)p.k_target : ceil(lam + 4.0 * sqrt(lam) + 8.0);
-    r = rr > (double)M ? (u32)M + 1u : (u32)rr;
-  }
+  // Ranks to read off the sample.  The number of sample points above a quantile is close to Poisson
+  // with mean lam, so "mean plus four standard deviations plus a constant" is almost never short.
+  const double lam_lo = (double)p.k_target * (double)M / (double)p.d;
+  const double lam_k = (double)p.k * (double)M / (double)p.d;
+  const bool exact = (int64_t)M == p.d;
+  const double r_lo_d = exact ? (double)p.k_target : ceil(lam_lo + 4.0 * sqrt(lam_lo) + 8.0);
+  const double r_hi_d = exact ? (double)p.k : floor(lam_k - 4.0 * sqrt(lam_k) - 8.0);
+  const u32 r_lo = r_lo_d > (double)M ? (u32)M + 1u : (u32)r_lo_d;
+  const u32 r_hi = r_hi_d < 1.0 ? 1u : (u32)r_hi_d;
+
+  // upper end of the key range the select should resolve finely: the k-th largest score cannot
+  // exceed the k-th largest |a|, estimated from above by the sample's r_hi-th largest
+  block_find_from_top(s_hist, kBins, r_hi, s_scan, s_res);
+  u32 hi_key = s_res[0] == kFull ? 0x7F7FFFFFu : (((s_res[0] + 1u) << 19) - 1u);
+  __syncthreads();
+  if (r_hi_d < 1.0) hi_key = hi_key < 0x7F000000u ? hi_key + (1u << 23) : 0x7F7FFFFFu;  // an octave of slack
+
   u32 cutoff = 0;
-  if (r <= (u32)M) {
-    block_find_from_top(s_hist, 4096, r, s_scan, s_res);
+  if (r_lo <= (u32)M) {
+    block_find_from_top(s_hist, kBins, r_lo, s_scan, s_res);
     const u32 b1 = s_res[0], above1 = s_res[1];
     __syncthreads();
     if (b1 != kFull) {
@@ -267,24 +299,25 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
       __syncthreads();
       for (int i = tid; i < nsect * 8; i += blockDim.x) {
         const u32 key = s_keys[i];
-        if ((key >> 19) == b1) {
-          // out-of-row sample slots hold key 0 and were not counted in level 1; keep them out
-          const int s = i >> 3, e = i & 7;
-          const int64_t q = all ? s : (int64_t)(((u64)s * (u64)Q) / (u64)kSampleSectors);
-          if (q * 8 + e < p.d) atomicAdd(&s_hist[(key >> 9) & 1023u], 1u);
-        }
+        if (key != kFull && (key >> 19) == b1) atomicAdd(&s_hist[(key >> 9) & 1023u], 1u);
       }
       __syncthreads();
-      block_find_from_top(s_hist, 1024, r - above1, s_scan, s_res);
+      block_find_from_top(s_hist, 1024, r_lo - above1, s_scan, s_res);
       const u32 b2 = s_res[0];
       cutoff = (b1 << 19) | ((b2 == kFull ? 0u : b2) << 9);
     }
   }
   if (tid == 0) {
-    p.ctl[n].cutoff = cutoff;
-    p.ctl[n].cand_count = 0;
-    p.ctl[n].state = kStateNormal;
-    p.ctl[n].n_valid = 0;
+    const u32 range = hi_key > cutoff ? hi_key - cutoff : 0u;
+    u32 shift = 0;
+    while ((range >> shift) > (u32)(kBins - 2)) ++shift;
+    ctl->cutoff = cutoff;
+    ctl->bin_shift = shift;
+    ctl->cand_count = 0;
+    ctl->force_dense = 0;
+    ctl->bcount = 0;
+    ctl->acount = 0;
+    ctl->n_valid = 0;
   }
 }
 
@@ -407,262 +440,140 @@ __global__ void __launch_bounds__(kStreamThreads) k_stream(StreamArgs p) {
   if (cur_n >= 0) stream_flush(list, wcount, p.ctl + cur_n, p.cand + (size_t)cur_n * p.stride, p.cap, lane);
 }
 
+
 // ---------------------------------------------------------------------------------------------
-// k_override: regularised scores on the previous support (Eq. (Delta_def), Algorithm 2 step 9).
+// cluster-wide helpers (every block of the cluster calls them, the same number of times)
 // ---------------------------------------------------------------------------------------------
-struct OverrideArgs {
-  const float* eps;  // holds a after k_stream
+struct PostShared {
+  u32 hist[kBins];     // this block's histogram; peers read it through distributed shared memory
+  u32 merged[kBins];   // this block's slice of the cluster-wide histogram
+  u32 tot[kMaxCluster];
+  u32 xch[kMaxCluster];
+  u32 res[2];
+  u32 fres[3];
+  u32 scan[33];
+  u32 cnt;
+};
+
+struct FindResult {
+  u32 bin, above, total;
+};
+
+// The blocks of a cluster have each filled sh.hist (kBins bins).  Returns, in every block, the bin of
+// the merged histogram that holds the r-th entry counted from the top, the entries above it, and the
+// grand total; bin == kFull if the total is below r.  Three cluster barriers.
+__device__ FindResult cluster_find_from_top(cg::cluster_group& cl, PostShared& sh, u32 r) {
+  const u32 CS = cl.num_blocks(), rk = cl.block_rank();
+  const int per = kBins / (int)CS;
+  const int tid = threadIdx.x;
+  cl.sync();  // all local histograms complete
+  u32 part = 0;
+  for (int b = tid; b < per; b += blockDim.x) {
+    const int bin = (int)rk * per + b;
+    u32 sum = 0;
+    for (u32 c = 0; c < CS; ++c) sum += cl.map_shared_rank(sh.hist, c)[bin];
+    sh.merged[b] = sum;
+    part += sum;
+  }
+  u32 slice_total;
+  block_excl_scan(part, sh.scan, &slice_total);
+  if (tid < (int)CS) cl.map_shared_rank(sh.tot, tid)[rk] = slice_total;
+  if (tid == 0) sh.res[0] = kFull;
+  cl.sync();  // slice totals delivered; every peer has finished reading this block's histogram
+  u32 acc = 0, total = 0;
+  int q = -1;
+  for (int s = (int)CS - 1; s >= 0; --s) {
+    const u32 t = sh.tot[s];
+    if (q < 0 && acc + t >= r) q = s;
+    if (q < 0) acc += t;
+    total += t;
+  }
+  if (q == (int)rk) {  // block-uniform
+    block_find_from_top(sh.merged, per, r - acc, sh.scan, sh.fres);
+    if (tid < (int)CS) {
+      u32* dst = cl.map_shared_rank(sh.res, tid);
+      dst[0] = sh.fres[0] == kFull ? kFull : (u32)((int)rk * per) + sh.fres[0];
+      dst[1] = acc + sh.fres[1];
+    }
+  }
+  cl.sync();  // result delivered
+  FindResult out;
+  out.bin = sh.res[0];
+  out.above = sh.res[1];
+  out.total = total;
+  return out;
+}
+
+// Exclusive prefix of one value per block over the cluster's block ranks, and the total.  Two barriers.
+__device__ u32 cluster_excl_sum(cg::cluster_group& cl, PostShared& sh, u32 v, u32* total) {
+  const u32 CS = cl.num_blocks(), rk = cl.block_rank();
+  if (threadIdx.x < CS) cl.map_shared_rank(sh.xch, threadIdx.x)[rk] = v;
+  cl.sync();
+  u32 pre = 0, tot = 0;
+  for (u32 c = 0; c < CS; ++c) {
+    const u32 t = sh.xch[c];
+    if (c < rk) pre += t;
+    tot += t;
+  }
+  *total = tot;
+  cl.sync();  // everyone has read; the exchange array may be written again
+  return pre;
+}
+
+__device__ __forceinline__ u32 warp_reserve_global(bool pred, u32* counter) {
+  const u32 m = __ballot_sync(kFull, pred);
+  if (m == 0) return 0;
+  const int lane = threadIdx.x & 31;
+  const int leader = __ffs(m) - 1;
+  u32 base = 0;
+  if (lane == leader) base = atomicAdd(counter, (u32)__popc(m));
+  base = __shfl_sync(kFull, base, leader);
+  return base + (u32)__popc(m & ((1u << lane) - 1u));
+}
+
+// ---------------------------------------------------------------------------------------------
+// k_post: one cluster per worker.
+// ---------------------------------------------------------------------------------------------
+struct PostArgs {
+  WorkerCtl* ctl;
+  GlobalCtl* gctl;
+  float* eps;  // holds a after k_stream; winners are zeroed here
   int64_t ld;
+  int64_t d;
+  int64_t k;
   const float* g_prev;
   const int32_t* prev_idx;
   const float* prev_val;
   const float* omega;
   float mu;
-  int64_t k;
-  int N;
-  const WorkerCtl* ctl;
   u32* ovr_key;   // [N][k] score bits of every previous-support entry
   u64* ovr_comp;  // [N][k] composite if the score reaches the cutoff, else 0
-};
-
-__global__ void __launch_bounds__(256) k_override(OverrideArgs p) {
-  const int64_t total = p.k * p.N;
-  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
-       t += (int64_t)gridDim.x * blockDim.x) {
-    const int n = (int)(t / p.k);
-    const int32_t j = p.prev_idx[t];
-    const float ap = p.prev_val[t];
-    const float G = p.g_prev[j];
-    const float a = p.eps[(size_t)n * p.ld + j];
-    const float w = p.omega[n];
-    const float num = __fsub_rn(G, __fmul_rn(w, ap));
-    const float den = __fmul_rn(w, a);
-    float m = 1.0f;
-    if (den != 0.0f) {
-      const float delta = __fdiv_rn(num, den);
-      const float r = fabsf(__fadd_rn(1.0f, delta));
-      m = tanh_fixed(__fdiv_rn(r, p.mu));
-    }
-    const u32 key = __float_as_uint(__fmul_rn(fabsf(a), m));
-    p.ovr_key[t] = key;
-    p.ovr_comp[t] = key >= p.ctl[n].cutoff ? make_composite(key, (u32)j) : 0ull;
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// k_select: one block per worker; exact k largest composites among candidates and overrides.
-// ---------------------------------------------------------------------------------------------
-struct SelectArgs {
-  WorkerCtl* ctl;
-  GlobalCtl* gctl;
-  u64* candA;        // [N][stride]; the stream pass fills at most capA entries of a row
+  u64* candA;     // [N][stride]; k_stream filled at most capA entries of a row
+  u64* candB;     // [N][stride]
   int64_t capA;
-  u64* candB;        // [N][stride]
-  int64_t stride;    // capA + k: what one histogram bin can hold (all candidates plus all overrides)
-  const u64* ovr_comp;
-  const int32_t* prev_idx;
-  u32* bitmask;      // [N][W]
-  int64_t W;
-  u32* tcount;       // [N][ntiles]
-  u32* toff;         // [N][ntiles]
-  int ntiles;
-  int64_t k;
-  int use_marks;     // previous support carries regularised scores (round >= 1, mu > 0)
-  int has_prev;      // bitmask holds last round's mask, to be cleared
-  int phase;         // 0: normal workers; 1: workers finished by the dense path
+  int64_t stride;  // capA + k: what one histogram bin can hold (all candidates plus all overrides)
+  u32* bitmask;    // [N][W] winners of this round (last round's on entry)
+  u32* wprefix;    // [N][W] winners before each non-empty mask word (rank directory for k_aggregate)
+  int64_t W;       // words per row, a multiple of 32
+  int32_t* out_idx;
+  float* out_val;
+  int32_t* cur_idx;
+  float* cur_val;
+  int use_marks;  // previous support carries regularised scores (round >= 1, mu > 0)
+  int has_prev;   // the bitmask holds last round's mask, to be cleared
 };
 
-__device__ __forceinline__ void set_winner(const SelectArgs& p, int n, u32 idx) {
-  atomicOr(&p.bitmask[(size_t)n * p.W + (idx >> 5)], 1u << (idx & 31));
-  atomicAdd(&p.tcount[(size_t)n * p.ntiles + (idx >> kTileShift)], 1u);
+__device__ __forceinline__ void set_winner(u32* mask, u32 idx) {
+  atomicOr(&mask[idx >> 5], 1u << (idx & 31));
 }
 
-__global__ void __launch_bounds__(kBlockSel) k_select(SelectArgs p) {
-  __shared__ u32 s_hist[4096];
-  __shared__ u32 s_scan[33];
-  __shared__ u32 s_res[3];
-  __shared__ u32 s_cnt;
-  const int n = blockIdx.x, tid = threadIdx.x;
-  WorkerCtl* ctl = p.ctl + n;
-  const u32 state = ctl->state;
-  if (p.phase == 0 ? state != kStateNormal : state != kStateDenseDone) return;
-
-  u64* A = p.candA + (size_t)n * p.stride;
-  u64* B = p.candB + (size_t)n * p.stride;
-  const u64* O = p.ovr_comp + (size_t)n * p.k;
-  const int32_t* prev_idx = p.prev_idx + (size_t)n * p.k;
-  u32* mask = p.bitmask + (size_t)n * p.W;
-  const u32 cand_count = ctl->cand_count;
-  const bool dense_done = p.phase == 1;
-  const bool use_marks = p.use_marks && !dense_done;
-  const u32 ncand = (u64)cand_count <= (u64)p.capA ? cand_count : (u32)p.capA;
-  const u32 novr = use_marks ? (u32)p.k : 0u;
-  const u32 k = (u32)p.k;
-
-  u32 need = k;
-  u32 nsrc = 0;
-  if (!dense_done) {
-    // filter: drop candidates that lie on the previous support (their score is the override's),
-    // histogram the top 12 key bits of everything valid
-    for (int i = tid; i < 4096; i += blockDim.x) s_hist[i] = 0;
-    __syncthreads();
-    for (u32 i = tid; i < ncand; i += blockDim.x) {
-      u64 c = A[i];
-      if (use_marks) {
-        const u32 idx = composite_idx(c);
-        if ((mask[idx >> 5] >> (idx & 31)) & 1u) {
-          A[i] = 0ull;
-          continue;
-        }
-      }
-      atomicAdd(&s_hist[(u32)(c >> 51)], 1u);
-    }
-    for (u32 i = tid; i < novr; i += blockDim.x) {
-      const u64 c = O[i];
-      if (c) atomicAdd(&s_hist[(u32)(c >> 51)], 1u);
-    }
-    __syncthreads();
-    block_find_from_top(s_hist, 4096, k, s_scan, s_res);
-    const u32 b1 = s_res[0], above1 = s_res[1], nvalid = s_res[2];
-    __syncthreads();
-    if (b1 == kFull || (u64)cand_count > (u64)p.capA) {
-      // too few valid candidates (cutoff guessed too high) or the list overflowed: dense path
-      if (tid == 0) {
-        ctl->state = kStateNeedDense;
-        ctl->n_valid = nvalid;
-        atomicAdd(&p.gctl->dense_workers, 1ull);
-      }
-      return;
-    }
-    if (tid == 0) {
-      ctl->n_valid = nvalid;
-      s_cnt = 0;
-    }
-    // every probe of the old mask is done: clear it (whole words; all their bits are old marks)
-    if (p.has_prev)
-      for (u32 i = tid; i < k; i += blockDim.x) mask[(u32)prev_idx[i] >> 5] = 0u;
-    __syncthreads();
-    // classify: above the bin -> winner; inside the bin -> list B for refinement
-    const u32 iters = (ncand + novr + blockDim.x - 1) / blockDim.x;
-    for (u32 it = 0; it < iters; ++it) {
-      const u32 i = it * blockDim.x + tid;
-      u64 c = 0ull;
-      if (i < ncand) c = A[i];
-      else if (i < ncand + novr) c = O[i - ncand];
-      const u32 bin = (u32)(c >> 51);
-      if (c && bin > b1) set_winner(p, n, composite_idx(c));
-      const bool inbin = c && bin == b1;
-      const u32 pos = warp_reserve(inbin, &s_cnt);
-      if (inbin) B[pos] = c;
-    }
-    __syncthreads();
-    need = k - above1;
-    nsrc = s_cnt;
-    __syncthreads();
-  } else {
-    // the dense path left exactly k winners in A
-    if (p.has_prev)
-      for (u32 i = tid; i < k; i += blockDim.x) mask[(u32)prev_idx[i] >> 5] = 0u;
-    __syncthreads();
-    need = k;
-    nsrc = k;
-    u64* t = A; A = B; B = t;  // so that "src" below is the list with the winners
-  }
-
-  // refinement on the remaining 51 composite bits, 8 at a time; src/dst ping-pong between B and A
-  u64* src = B;
-  u64* dst = A;
-  int shift = 43;
-  while (true) {
-    if (need == 0) break;
-    if (need == nsrc) {
-      for (u32 i = tid; i < nsrc; i += blockDim.x) set_winner(p, n, composite_idx(src[i]));
-      break;
-    }
-    if (shift < -8) {  // all 51 bits consumed and still undecided: composites were not unique
-      if (tid == 0) atomicOr(&p.gctl->err, kErrCountMismatch);
-      break;
-    }
-    const int sh = shift >= 0 ? shift : 0;
-    const u32 dmask = shift >= 0 ? 255u : 7u;  // the last digit is the low 3 bits
-    for (int i = tid; i < 256; i += blockDim.x) s_hist[i] = 0;
-    if (tid == 0) s_cnt = 0;
-    __syncthreads();
-    for (u32 i = tid; i < nsrc; i += blockDim.x) atomicAdd(&s_hist[(u32)(src[i] >> sh) & dmask], 1u);
-    __syncthreads();
-    block_find_from_top(s_hist, 256, need, s_scan, s_res);
-    const u32 b = s_res[0], above = s_res[1];
-    __syncthreads();
-    if (b == kFull) {  // cannot happen: need <= nsrc
-      if (tid == 0) atomicOr(&p.gctl->err, kErrCountMismatch);
-      break;
-    }
-    const u32 iters = (nsrc + blockDim.x - 1) / blockDim.x;
-    for (u32 it = 0; it < iters; ++it) {
-      const u32 i = it * blockDim.x + tid;
-      u64 c = 0ull;
-      u32 dg = 0;
-      if (i < nsrc) {
-        c = src[i];
-        dg = (u32)(c >> sh) & dmask;
-        if (dg > b) set_winner(p, n, composite_idx(c));
-      }
-      const bool inbin = i < nsrc && dg == b;
-      const u32 pos = warp_reserve(inbin, &s_cnt);
-      if (inbin) dst[pos] = c;
-    }
-    __syncthreads();
-    need -= above;
-    nsrc = s_cnt;
-    __syncthreads();
-    u64* t = src; src = dst; dst = t;
-    shift -= 8;
-  }
-  __syncthreads();
-  __threadfence_block();
-
-  // exclusive scan of the per-tile winner counts -> output offsets of k_emit
-  {
-    u32* tc = p.tcount + (size_t)n * p.ntiles;
-    u32* to = p.toff + (size_t)n * p.ntiles;
-    const int per = (p.ntiles + blockDim.x - 1) / blockDim.x;
-    const int first = tid * per;
-    u32 sum = 0;
-    for (int i = 0; i < per; ++i)
-      if (first + i < p.ntiles) sum += __ldcg(tc + first + i);
-    u32 total;
-    u32 run = block_excl_scan(sum, s_scan, &total);
-    for (int i = 0; i < per; ++i)
-      if (first + i < p.ntiles) {
-        to[first + i] = run;
-        run += __ldcg(tc + first + i);
-      }
-    if (tid == 0 && total != k) atomicOr(&p.gctl->err, kErrCountMismatch);
-  }
+__device__ __forceinline__ u32 select_bin(u32 key, u32 cutoff, u32 shift) {
+  const u32 b = (key - cutoff) >> shift;
+  return b < (u32)(kBins - 1) ? b : (u32)(kBins - 1);
 }
 
-// ---------------------------------------------------------------------------------------------
-// k_dense_select: exact selection over the whole row for workers in state NeedDense.  One block per
-// worker; slow (every pass walks d entries with 1024 threads) but right for any input, including
-// rows of equal values.  Leaves the k winners in the worker's candidate list A.
-// ---------------------------------------------------------------------------------------------
-struct DenseArgs {
-  WorkerCtl* ctl;
-  GlobalCtl* gctl;
-  const float* eps;  // holds a
-  int64_t ld;
-  int64_t d;
-  int64_t k;
-  const u32* bitmask;
-  int64_t W;
-  const int32_t* prev_idx;
-  const u32* ovr_key;
-  u64* candA;
-  int64_t stride;
-  int use_marks;
-};
-
-__device__ __forceinline__ u32 dense_key(const DenseArgs& p, int n, int64_t j) {
+// Score key of entry j for the dense path: the override's on the previous support, bits(|a|) elsewhere.
+__device__ __forceinline__ u32 dense_key(const PostArgs& p, int n, int64_t j) {
   if (p.use_marks) {
     const u32 w = p.bitmask[(size_t)n * p.W + (j >> 5)];
     if ((w >> (j & 31)) & 1u) {
@@ -678,185 +589,380 @@ __device__ __forceinline__ u32 dense_key(const DenseArgs& p, int n, int64_t j) {
   return __float_as_uint(p.eps[(size_t)n * p.ld + j]) & 0x7FFFFFFFu;
 }
 
-__global__ void __launch_bounds__(kBlockSel) k_dense_select(DenseArgs p) {
-  __shared__ u32 s_hist[4096];
-  __shared__ u32 s_scan[33];
-  __shared__ u32 s_res[3];
-  __shared__ u32 s_cnt;
-  const int n = blockIdx.x, tid = threadIdx.x;
-  WorkerCtl* ctl = p.ctl + n;
-  if (ctl->state != kStateNeedDense) return;
-  u64* A = p.candA + (size_t)n * p.stride;
-
-  u32 need = (u32)p.k;
-  u32 prefix = 0;
-  // three digits of the 31-bit key: bits 30..19, 18..7, 6..0
-  const int shifts[3] = {19, 7, 0};
-  const int widths[3] = {12, 12, 7};
-  for (int lv = 0; lv < 3; ++lv) {
-    const int sh = shifts[lv], nb = 1 << widths[lv];
-    for (int i = tid; i < nb; i += blockDim.x) s_hist[i] = 0;
+// Leader block only: pick the `need` largest composites of list[0..count) and set them as winners.
+// Uses `other` (same capacity) as the second buffer of the radix passes.
+__device__ void refine_list(PostShared& sh, u32* mask, GlobalCtl* gctl, u64* list, u64* other,
+                            u32 count, u32 need) {
+  const int tid = threadIdx.x;
+  if (need == 0) return;
+  if (need >= count) {
+    for (u32 i = tid; i < count; i += blockDim.x) set_winner(mask, composite_idx(list[i]));
+    return;
+  }
+  if (count <= (u32)kBins) {
+    // small list: rank every item by counting the items above it (composites are unique)
+    u64* s_items = reinterpret_cast<u64*>(sh.hist);  // hist and merged are contiguous: kBins u64
+    for (u32 i = tid; i < count; i += blockDim.x) s_items[i] = list[i];
     __syncthreads();
-    for (int64_t j = tid; j < p.d; j += blockDim.x) {
-      const u32 key = dense_key(p, n, j);
-      if (lv == 0 || (key >> (sh + widths[lv])) == prefix) atomicAdd(&s_hist[(key >> sh) & (nb - 1)], 1u);
+    for (u32 i = tid; i < count; i += blockDim.x) {
+      const u64 c = s_items[i];
+      u32 above = 0;
+      for (u32 j = 0; j < count; ++j) above += s_items[j] > c ? 1u : 0u;
+      if (above < need) set_winner(mask, composite_idx(c));
     }
     __syncthreads();
-    block_find_from_top(s_hist, nb, need, s_scan, s_res);
-    const u32 b = s_res[0], above = s_res[1];
+    return;
+  }
+  // general case (long runs of equal keys): radix passes over all 64 composite bits
+  u64* src = list;
+  u64* dst = other;
+  u32 nsrc = count;
+  for (int shift = 56; shift >= 0; shift -= 8) {
+    if (need == 0) return;
+    if (need == nsrc) break;
+    for (int i = tid; i < 256; i += blockDim.x) sh.hist[i] = 0;
+    if (tid == 0) sh.cnt = 0;
     __syncthreads();
-    if (b == kFull) {
-      if (tid == 0) atomicOr(&p.gctl->err, kErrDenseSelect);
+    for (u32 i = tid; i < nsrc; i += blockDim.x) atomicAdd(&sh.hist[(u32)(src[i] >> shift) & 255u], 1u);
+    __syncthreads();
+    block_find_from_top(sh.hist, 256, need, sh.scan, sh.fres);
+    const u32 b = sh.fres[0], above = sh.fres[1];
+    __syncthreads();
+    if (b == kFull) {  // cannot happen: need <= nsrc
+      if (tid == 0) atomicOr(&gctl->err, kErrRefine);
       return;
     }
-    need -= above;
-    prefix = (prefix << widths[lv]) | b;
-  }
-  const u32 T = prefix;                   // key of the k-th largest score
-  const u32 n_gt = (u32)p.k - need;       // entries strictly above it; `need` ties are to be taken
-  if (tid == 0) s_cnt = 0;
-  __syncthreads();
-  // entries above T, in any order
-  for (int64_t base = 0; base < p.d; base += blockDim.x) {
-    const int64_t j = base + tid;
-    u32 key = 0;
-    bool gt = false;
-    if (j < p.d) {
-      key = dense_key(p, n, j);
-      gt = key > T;
-    }
-    const u32 pos = warp_reserve(gt, &s_cnt);
-    if (gt && pos < n_gt) A[pos] = make_composite(key, (u32)j);
-  }
-  __syncthreads();
-  if (tid == 0 && s_cnt != n_gt) atomicOr(&p.gctl->err, kErrDenseSelect);
-  // ties in index order: the first `need` of them
-  u32 taken = 0;
-  for (int64_t base = 0; base < p.d && taken < need; base += blockDim.x) {
-    const int64_t j = base + tid;
-    const bool tie = j < p.d && dense_key(p, n, j) == T;
-    u32 total;
-    const u32 rank = taken + block_excl_scan(tie ? 1u : 0u, s_scan, &total);
-    if (tie && rank < need) A[n_gt + rank] = make_composite(T, (u32)j);
-    taken += total;
-  }
-  if (tid == 0) {
-    if (taken < need) atomicOr(&p.gctl->err, kErrDenseSelect);
-    ctl->cand_count = (u32)p.k;
-    ctl->state = kStateDenseDone;
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// k_emit: ordered walk of the winner bitmask.  One block per (tile, worker); ascending indices.
-// ---------------------------------------------------------------------------------------------
-struct EmitArgs {
-  const u32* bitmask;
-  int64_t W;
-  const u32* tcount;
-  const u32* toff;
-  int ntiles;
-  float* eps;
-  int64_t ld;
-  int64_t k;
-  int32_t* out_idx;
-  float* out_val;
-  int32_t* cur_idx;
-  float* cur_val;
-};
-
-__global__ void __launch_bounds__(256) k_emit(EmitArgs p) {
-  __shared__ u32 s_scan[33];
-  const int t = blockIdx.x, n = blockIdx.y, tid = threadIdx.x;
-  if (p.tcount[(size_t)n * p.ntiles + t] == 0) return;
-  const u32* words = p.bitmask + (size_t)n * p.W + (size_t)t * kTileWords + tid * 8;
-  const uint4 w0 = *reinterpret_cast<const uint4*>(words);
-  const uint4 w1 = *reinterpret_cast<const uint4*>(words + 4);
-  u32 w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-  u32 c = 0;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) c += __popc(w[i]);
-  u32 total;
-  u32 pos = p.toff[(size_t)n * p.ntiles + t] + block_excl_scan(c, s_scan, &total);
-  if (c == 0) return;
-  float* eps_row = p.eps + (size_t)n * p.ld;
-  const size_t obase = (size_t)n * p.k;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    u32 bits = w[i];
-    const u32 jbase = ((u32)t * kTileWords + tid * 8 + i) << 5;
-    while (bits) {
-      const int b = __ffs(bits) - 1;
-      bits &= bits - 1;
-      const u32 j = jbase + b;
-      const float v = eps_row[j];
-      eps_row[j] = 0.0f;  // a - a
-      if (pos < (u32)p.k) {  // always true when the tile counts are consistent
-        p.out_idx[obase + pos] = (int32_t)j;
-        p.out_val[obase + pos] = v;
-        p.cur_idx[obase + pos] = (int32_t)j;
-        p.cur_val[obase + pos] = v;
+    const u32 iters = (nsrc + blockDim.x - 1) / blockDim.x;
+    for (u32 it = 0; it < iters; ++it) {
+      const u32 i = it * blockDim.x + tid;
+      u64 c = 0ull;
+      u32 dg = 0;
+      if (i < nsrc) {
+        c = src[i];
+        dg = (u32)(c >> shift) & 255u;
+        if (dg > b) set_winner(mask, composite_idx(c));
       }
-      ++pos;
+      const bool inbin = i < nsrc && dg == b;
+      const u32 pos = warp_reserve(inbin, &sh.cnt);
+      if (inbin) dst[pos] = c;
     }
+    __syncthreads();
+    need -= above;
+    nsrc = sh.cnt;
+    __syncthreads();
+    u64* t = src; src = dst; dst = t;
+  }
+  if (need == nsrc) {
+    for (u32 i = tid; i < nsrc; i += blockDim.x) set_winner(mask, composite_idx(src[i]));
+  } else if (need != 0) {
+    if (tid == 0) atomicOr(&gctl->err, kErrRefine);  // all bits consumed: composites were not unique
   }
 }
 
+__global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
+  __shared__ __align__(16) PostShared sh;
+  cg::cluster_group cl = cg::this_cluster();
+  const u32 CS = cl.num_blocks(), rk = cl.block_rank();
+  const int n = blockIdx.x / CS;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const u32 stride_t = CS * blockDim.x;        // threads of the cluster
+  const u32 first_t = rk * blockDim.x + tid;   // this thread's index among them
+  WorkerCtl* ctl = p.ctl + n;
+  const u32 cutoff = ctl->cutoff, bshift = ctl->bin_shift;
+  const u32 cand_count = ctl->cand_count;
+  bool dense = ctl->force_dense != 0;          // identical in every block: nothing writes it here
+  const u32 k = (u32)p.k;
+  u64* A = p.candA + (size_t)n * p.stride;
+  u64* B = p.candB + (size_t)n * p.stride;
+  u64* O = p.ovr_comp + (size_t)n * p.k;
+  u32* okey = p.ovr_key + (size_t)n * p.k;
+  const int32_t* prev_idx = p.prev_idx + (size_t)n * p.k;
+  const float* prev_val = p.prev_val + (size_t)n * p.k;
+  u32* mask = p.bitmask + (size_t)n * p.W;
+  u32* wpre = p.wprefix + (size_t)n * p.W;
+  float* eps_row = p.eps + (size_t)n * p.ld;
+  const bool overflow = (u64)cand_count > (u64)p.capA;
+  const u32 ncand = overflow ? (u32)p.capA : cand_count;
+  const u32 novr = p.use_marks ? k : 0u;
+
+  // ---- regularised scores on the previous support (Eq. (Delta_def), Algorithm 2 step 9) ----
+  if (p.use_marks) {
+    const float w = p.omega[n];
+    for (u32 i = first_t; i < k; i += stride_t) {
+      const int32_t j = prev_idx[i];
+      const float a = eps_row[j];
+      const float num = __fsub_rn(p.g_prev[j], __fmul_rn(w, prev_val[i]));
+      const float den = __fmul_rn(w, a);
+      float m = 1.0f;
+      if (den != 0.0f) {
+        const float delta = __fdiv_rn(num, den);
+        const float r = fabsf(__fadd_rn(1.0f, delta));
+        m = tanh_fixed(__fdiv_rn(r, p.mu));
+      }
+      const u32 key = __float_as_uint(__fmul_rn(fabsf(a), m));
+      okey[i] = key;
+      O[i] = key >= cutoff ? make_composite(key, (u32)j) : 0ull;
+    }
+  }
+  for (int i = tid; i < kBins; i += blockDim.x) sh.hist[i] = 0;
+  cl.sync();  // override keys visible to the whole cluster; histograms cleared
+
+  FindResult fr;
+  fr.bin = kFull; fr.above = 0; fr.total = 0;
+  if (!dense) {
+    // ---- filter and histogram: candidates on the previous support are dropped (their score is the
+    //      override's); every thread keeps the same items in the later classify pass ----
+    for (u32 i = first_t; i < ncand; i += stride_t) {
+      const u64 c = A[i];
+      if (p.use_marks) {
+        const u32 idx = composite_idx(c);
+        if ((mask[idx >> 5] >> (idx & 31)) & 1u) {
+          A[i] = 0ull;
+          continue;
+        }
+      }
+      atomicAdd(&sh.hist[select_bin((u32)(c >> 32), cutoff, bshift)], 1u);
+    }
+    for (u32 i = first_t; i < novr; i += stride_t) {
+      const u64 c = O[i];
+      if (c) atomicAdd(&sh.hist[select_bin((u32)(c >> 32), cutoff, bshift)], 1u);
+    }
+    fr = cluster_find_from_top(cl, sh, k);
+    if (fr.bin == kFull || overflow) dense = true;  // cutoff guessed too high, or the list overflowed
+    if (rk == 0 && tid == 0) ctl->n_valid = fr.total;
+  }
+
+  if (!dense) {
+    // every probe of the old mask is done: clear it (whole words; all their bits are old marks)
+    if (p.has_prev)
+      for (u32 i = first_t; i < k; i += stride_t) mask[(u32)prev_idx[i] >> 5] = 0u;
+    cl.sync();
+    // ---- classify: above the bin -> winner; inside it -> refinement list ----
+    const u32 total_items = ncand + novr;
+    const u32 iters = (total_items + stride_t - 1) / stride_t;
+    for (u32 it = 0; it < iters; ++it) {
+      const u32 i = it * stride_t + first_t;
+      u64 c = 0ull;
+      if (i < ncand) c = A[i];
+      else if (i < total_items) c = O[i - ncand];
+      const u32 bin = c ? select_bin((u32)(c >> 32), cutoff, bshift) : 0u;
+      if (c && bin > fr.bin) set_winner(mask, composite_idx(c));
+      const bool inbin = c && bin == fr.bin;
+      const u32 pos = warp_reserve_global(inbin, &ctl->bcount);
+      if (inbin) B[pos] = c;
+    }
+    cl.sync();
+    if (rk == 0) refine_list(sh, mask, p.gctl, B, A, __ldcg(&ctl->bcount), k - fr.above);
+  } else {
+    // ---- exact selection over the whole row: three radix digits of the 31-bit key ----
+    if (rk == 0 && tid == 0) atomicAdd(&p.gctl->dense_workers, 1ull);
+    const int64_t c0 = (int64_t)(((u64)rk * (u64)p.d) / CS);
+    const int64_t c1 = (int64_t)(((u64)(rk + 1) * (u64)p.d) / CS);
+    u32 need = k, prefix = 0;
+    bool bad = false;
+    const int shifts[3] = {19, 7, 0};
+    const int widths[3] = {12, 12, 7};
+    for (int lv = 0; lv < 3; ++lv) {
+      const int shf = shifts[lv];
+      const u32 nbm = (1u << widths[lv]) - 1u;
+      __syncthreads();
+      for (int i = tid; i < kBins; i += blockDim.x) sh.hist[i] = 0;
+      __syncthreads();
+      for (int64_t j = c0 + tid; j < c1; j += blockDim.x) {
+        const u32 key = dense_key(p, n, j);
+        if (lv == 0 || (key >> (shf + widths[lv])) == prefix) atomicAdd(&sh.hist[(key >> shf) & nbm], 1u);
+      }
+      const FindResult r = cluster_find_from_top(cl, sh, need);
+      if (r.bin == kFull) bad = true;
+      const u32 b = r.bin == kFull ? 0u : r.bin;
+      need -= r.bin == kFull ? 0u : r.above;
+      prefix = (prefix << widths[lv]) | b;
+    }
+    const u32 T = prefix;          // key of the k-th largest score
+    const u32 n_gt = k - need;     // entries strictly above it; `need` ties are to be taken
+    // entries above T in any order, and this block's count of ties
+    u32 my_ties = 0;
+    for (int64_t base = c0; base < c1; base += blockDim.x) {
+      const int64_t j = base + tid;
+      u32 key = 0;
+      bool gt = false;
+      if (j < c1) {
+        key = dense_key(p, n, j);
+        gt = key > T;
+        my_ties += key == T ? 1u : 0u;
+      }
+      const u32 pos = warp_reserve_global(gt, &ctl->acount);
+      if (gt && pos < n_gt) A[pos] = make_composite(key, (u32)j);
+    }
+    u32 block_ties;
+    block_excl_scan(my_ties, sh.scan, &block_ties);
+    u32 all_ties;
+    u32 taken = cluster_excl_sum(cl, sh, block_ties, &all_ties);  // ties in lower-index blocks
+    if (all_ties < need) bad = true;
+    // ties in index order: the first `need` of them
+    for (int64_t base = c0; base < c1 && taken < need; base += blockDim.x) {
+      const int64_t j = base + tid;
+      const bool tie = j < c1 && dense_key(p, n, j) == T;
+      u32 total;
+      const u32 rank = taken + block_excl_scan(tie ? 1u : 0u, sh.scan, &total);
+      if (tie && rank < need) A[n_gt + rank] = make_composite(T, (u32)j);
+      taken += total;
+    }
+    cl.sync();  // winner list complete; nobody reads the old mask any more
+    if (rk == 0 && tid == 0 && (bad || __ldcg(&ctl->acount) != n_gt)) atomicOr(&p.gctl->err, kErrDenseSelect);
+    if (p.has_prev)
+      for (u32 i = first_t; i < k; i += stride_t) mask[(u32)prev_idx[i] >> 5] = 0u;
+    cl.sync();
+    if (!bad)
+      for (u32 i = first_t; i < k; i += stride_t) set_winner(mask, composite_idx(__ldcg(&A[i])));
+  }
+  cl.sync();  // every winner bit is set
+
+  // ---- emission: ordered walk of the bitmask; blocks and warps own contiguous ranges of 32-word groups ----
+  const int64_t G = p.W >> 5;
+  const int64_t g0 = (int64_t)(((u64)rk * (u64)G) / CS), g1 = (int64_t)(((u64)(rk + 1) * (u64)G) / CS);
+  const int nw = blockDim.x >> 5;
+  const int64_t wg0 = g0 + ((g1 - g0) * warp) / nw, wg1 = g0 + ((g1 - g0) * (warp + 1)) / nw;
+  u32 wsum = 0;
+  for (int64_t g = wg0; g < wg1; ++g) wsum += __popc(__ldcg(&mask[g * 32 + lane]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(kFull, wsum, o);
+  u32 block_total;
+  u32 warp_pre = block_excl_scan(lane == 0 ? wsum : 0u, sh.scan, &block_total);
+  warp_pre = __shfl_sync(kFull, warp_pre, 0);
+  u32 all_total;
+  const u32 block_pre = cluster_excl_sum(cl, sh, block_total, &all_total);
+  if (rk == 0 && tid == 0 && all_total != k) atomicOr(&p.gctl->err, kErrCountMismatch);
+  if (all_total == k) {
+    u32 running = block_pre + warp_pre;
+    const size_t obase = (size_t)n * p.k;
+    for (int64_t g = wg0; g < wg1; ++g) {
+      const u32 word = __ldcg(&mask[g * 32 + lane]);
+      const u32 c = __popc(word);
+      u32 inc = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const u32 t = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += t;
+      }
+      const u32 T = __shfl_sync(kFull, inc, 31);
+      if (T == 0) continue;
+      const u32 pre = inc - c;
+      if (word) wpre[g * 32 + lane] = running + pre;
+      // balanced extraction: rank r of the group belongs to lane r % 32, four ranks in flight
+      for (u32 r0 = 0; r0 < T; r0 += 128) {
+        u32 jj[4];
+        float vv[4];
+        bool act[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const u32 r = r0 + q * 32 + lane;
+          act[q] = r < T;
+          const u32 rr = act[q] ? r : T - 1;
+          u32 lo = 0;  // the last word whose exclusive prefix is <= rr holds rank rr
+#pragma unroll
+          for (int step = 16; step > 0; step >>= 1) {
+            const u32 cand = lo + step;
+            const u32 pc = __shfl_sync(kFull, pre, cand & 31);
+            if (cand < 32 && pc <= rr) lo = cand;
+          }
+          const u32 ww = __shfl_sync(kFull, word, lo);
+          const u32 pw = __shfl_sync(kFull, pre, lo);
+          const u32 bit = __fns(ww, 0, (int)(rr - pw) + 1);
+          jj[q] = (u32)((g * 32 + lo) << 5) + bit;
+          vv[q] = act[q] ? eps_row[jj[q]] : 0.0f;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (act[q]) {
+            const size_t o = obase + running + r0 + q * 32 + lane;
+            eps_row[jj[q]] = 0.0f;  // a - a
+            p.out_idx[o] = (int32_t)jj[q];
+            p.out_val[o] = vv[q];
+            p.cur_idx[o] = (int32_t)jj[q];
+            p.cur_val[o] = vv[q];
+          }
+        }
+      }
+      running += T;
+    }
+  }
+  cl.sync();  // no block leaves while a peer may still read its shared memory
+}
+
 // ---------------------------------------------------------------------------------------------
-// k_aggregate: g = sum_n omega_n * ghat_n in worker order.  The coordinate range is cut into
-// gridDim.x slices; a block owns a slice, so all updates of one coordinate happen in one block,
-// ordered by the barrier between workers.  Last round's entries are cleared first.
+// k_aggregate: g = sum_n omega_n * ghat_n with the workers added in the order n = 0..N-1.
+// One thread per pair sent this round: the pair of the highest-numbered worker that sent index j
+// owns g[j]; it looks the lower workers' values up (mask word, prefix count, value) and adds them
+// in order.  One thread per pair of the previous round clears g[j] if nobody sent j now.
 // ---------------------------------------------------------------------------------------------
 struct AggArgs {
   float* g;
-  int64_t d;
   int N;
   int64_t k;
   const int32_t* cur_idx;
   const float* cur_val;
   const int32_t* prev_idx;
+  const u32* bitmask;
+  const u32* wprefix;
+  int64_t W;
   const float* omega;
   int has_prev;
 };
 
-__device__ __forceinline__ int64_t lower_bound_i32(const int32_t* a, int64_t n, int64_t v) {
-  int64_t lo = 0, hi = n;
-  while (lo < hi) {
-    const int64_t mid = (lo + hi) >> 1;
-    if ((int64_t)a[mid] < v) lo = mid + 1; else hi = mid;
-  }
-  return lo;
-}
-
 __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
-  extern __shared__ int64_t s_bounds[];  // [2 lists][N][2]
-  const int tid = threadIdx.x;
-  const int64_t lo = (int64_t)(((u64)blockIdx.x * (u64)p.d) / gridDim.x);
-  const int64_t hi = (int64_t)(((u64)(blockIdx.x + 1) * (u64)p.d) / gridDim.x);
-  for (int t = tid; t < 4 * p.N; t += blockDim.x) {
-    const int list = t / (2 * p.N), n = (t >> 1) % p.N, side = t & 1;
-    const int32_t* arr = (list ? p.prev_idx : p.cur_idx) + (size_t)n * p.k;
-    s_bounds[t] = (list && !p.has_prev) ? 0 : lower_bound_i32(arr, p.k, side ? hi : lo);
-  }
-  __syncthreads();
-  if (p.has_prev) {
-    for (int n = 0; n < p.N; ++n) {
-      const int64_t b = s_bounds[2 * p.N + 2 * n], e = s_bounds[2 * p.N + 2 * n + 1];
-      const int32_t* pi = p.prev_idx + (size_t)n * p.k;
-      for (int64_t i = b + tid; i < e; i += blockDim.x) p.g[pi[i]] = 0.0f;
+  const int64_t npairs = p.k * p.N;
+  const int64_t total = p.has_prev ? 2 * npairs : npairs;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (int64_t)gridDim.x * blockDim.x) {
+    if (t >= npairs) {  // a pair of the previous round
+      const int32_t j = p.prev_idx[t - npairs];
+      const size_t wi = (size_t)(j >> 5);
+      const u32 bm = 1u << (j & 31);
+      u32 any = 0;
+      for (int m0 = 0; m0 < p.N; m0 += 8) {
+        u32 w[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) w[u] = m0 + u < p.N ? p.bitmask[(size_t)(m0 + u) * p.W + wi] : 0u;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) any |= w[u];
+      }
+      if (!(any & bm)) p.g[j] = 0.0f;
+      continue;
     }
-    __syncthreads();
-  }
-  for (int n = 0; n < p.N; ++n) {
-    const int64_t b = s_bounds[2 * n], e = s_bounds[2 * n + 1];
-    const int32_t* ci = p.cur_idx + (size_t)n * p.k;
-    const float* cv = p.cur_val + (size_t)n * p.k;
-    const float w = p.omega[n];
-    for (int64_t i = b + tid; i < e; i += blockDim.x) {
-      const int32_t j = ci[i];
-      p.g[j] = __fadd_rn(p.g[j], __fmul_rn(w, cv[i]));
+    const int n = (int)(t / p.k);
+    const int32_t j = p.cur_idx[t];
+    const size_t wi = (size_t)(j >> 5);
+    const u32 bm = 1u << (j & 31);
+    // a higher-numbered worker that sent j owns it
+    bool owned = true;
+    for (int m0 = n + 1; m0 < p.N && owned; m0 += 8) {
+      u32 w[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) w[u] = m0 + u < p.N ? p.bitmask[(size_t)(m0 + u) * p.W + wi] : 0u;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) owned = owned && !(w[u] & bm);
     }
-    __syncthreads();
+    if (!owned) continue;
+    float sum = 0.0f;
+    for (int m0 = 0; m0 < n; m0 += 8) {
+      u32 w[8], pre[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const bool in = m0 + u < n;
+        w[u] = in ? p.bitmask[(size_t)(m0 + u) * p.W + wi] : 0u;
+        pre[u] = in ? p.wprefix[(size_t)(m0 + u) * p.W + wi] : 0u;
+      }
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        v[u] = (w[u] & bm) ? p.cur_val[(size_t)(m0 + u) * p.k + pre[u] + __popc(w[u] & (bm - 1u))] : 0.0f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (w[u] & bm) sum = __fadd_rn(sum, __fmul_rn(p.omega[m0 + u], v[u]));
+    }
+    sum = __fadd_rn(sum, __fmul_rn(p.omega[n], p.cur_val[t]));
+    p.g[j] = sum;
   }
 }
 
@@ -866,11 +972,10 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  int64_t ld, W, capA, capB;
-  int ntiles;
-  size_t off_eps, off_g, off_mask, off_tcount, off_toff, off_idx[2], off_val[2], off_ovr_key,
-      off_ovr_comp, off_candA, off_candB, off_ctl, off_gctl, off_omega, off_stage_g, off_stage_idx,
-      off_stage_val, zero_end, total;
+  int64_t ld, W, capA, stride;
+  size_t off_eps, off_g, off_mask, off_ctl, off_gctl, zero_end, off_wprefix, off_idx[2], off_val[2],
+      off_ovr_key, off_ovr_comp, off_candA, off_candB, off_omega, off_stage_g, off_stage_idx,
+      off_stage_val, total;
 };
 
 bool valid_problem(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
@@ -887,34 +992,32 @@ bool valid_problem(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
 Layout make_layout(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
   Layout L;
   L.ld = (int64_t)align_up((size_t)d, 1024);
-  L.ntiles = (int)((d + (1 << kTileShift) - 1) >> kTileShift);
-  L.W = (int64_t)L.ntiles * kTileWords;
+  L.W = (int64_t)align_up((size_t)((d + 31) / 32), 32);
   const int64_t M = d < kSampleMax ? d : kSampleMax;
   const int64_t kt = pr->mu > 0.0f ? (2 * k < d ? 2 * k : d) : k;
   int64_t cap = 2 * kt + 64 * ((d + M - 1) / M) + 4096;
   if (cap > d) cap = d;
   if (cap < k) cap = k;
   L.capA = cap;
-  L.capB = cap + k;
+  L.stride = cap + k;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
   // state that creation and reset clear to zero comes first
   L.off_eps = take((size_t)N * L.ld * 4);
   L.off_g = take(align_up((size_t)d, 64) * 4);
   L.off_mask = take((size_t)N * L.W * 4);
-  L.off_tcount = take((size_t)N * L.ntiles * 4);
-  L.off_toff = take((size_t)N * L.ntiles * 4);
   L.off_ctl = take((size_t)N * sizeof(WorkerCtl));
   L.off_gctl = take(sizeof(GlobalCtl));
   L.zero_end = o;
+  L.off_wprefix = take((size_t)N * L.W * 4);
   for (int i = 0; i < 2; ++i) {
     L.off_idx[i] = take((size_t)N * k * 4);
     L.off_val[i] = take((size_t)N * k * 4);
   }
   L.off_ovr_key = take((size_t)N * k * 4);
   L.off_ovr_comp = take((size_t)N * k * 8);
-  L.off_candA = take((size_t)N * L.capB * 8);
-  L.off_candB = take((size_t)N * L.capB * 8);
+  L.off_candA = take((size_t)N * L.stride * 8);
+  L.off_candB = take((size_t)N * L.stride * 8);
   L.off_omega = take((size_t)N * 4);
   L.off_stage_g = L.off_stage_idx = L.off_stage_val = 0;
   if (pr->flags & REGTOPK_FLAG_HOST_STAGING) {
@@ -943,6 +1046,7 @@ struct regtopk_ctx {
   int stepped;       // worker_step done, aggregate pending
   int sticky;        // first CUDA error seen
   int num_sms;
+  int cluster;       // blocks per worker in k_post
   int stream_blocks[4];
   int64_t launches;
   int profiling;
@@ -967,7 +1071,7 @@ int after_launch(regtopk_ctx* c) {
   return note_cuda(c, cudaGetLastError());
 }
 
-size_t sample_smem() { return (size_t)(kSampleMax + 4096) * sizeof(u32); }
+size_t sample_smem() { return (size_t)(kSampleMax + kBins) * sizeof(u32); }
 
 template <bool BF16, bool VEC>
 void launch_stream(regtopk_ctx* c, const StreamArgs& a, int variant) {
@@ -981,6 +1085,38 @@ void launch_stream(regtopk_ctx* c, const StreamArgs& a, int variant) {
   int64_t blocks = (chunks + (kStreamThreads / 32) - 1) / (kStreamThreads / 32);
   if (blocks > c->stream_blocks[variant]) blocks = c->stream_blocks[variant];
   k_stream<BF16, VEC><<<(unsigned)blocks, kStreamThreads, 0, c->stream>>>(a);
+}
+
+void post_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int N, int cluster, cudaStream_t s) {
+  memset(cfg, 0, sizeof *cfg);
+  cfg->gridDim = dim3((unsigned)(N * cluster), 1, 1);
+  cfg->blockDim = dim3(kBlockSel, 1, 1);
+  cfg->dynamicSmemBytes = 0;
+  cfg->stream = s;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg->attrs = attr;
+  cfg->numAttrs = 1;
+}
+
+// Blocks per worker for k_post: as many as keep all N clusters resident at once, a power of two,
+// at most 16 (sizes above 8 need the non-portable opt-in), and only what the device can schedule.
+int choose_cluster(int N, int num_sms) {
+  int want = 16;
+  while (want > 1 && N * want > num_sms) want >>= 1;
+  cudaFuncSetAttribute(k_post, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  cudaGetLastError();
+  for (int cs = want; cs > 1; cs >>= 1) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    post_config(&cfg, attr, N, cs, nullptr);
+    int nclusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&nclusters, k_post, &cfg) == cudaSuccess && nclusters >= 1) return cs;
+    cudaGetLastError();
+  }
+  return 1;
 }
 
 }  // namespace
@@ -1045,6 +1181,7 @@ int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const reg
   c->ws = static_cast<char*>(workspace);
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->num_sms = sms > 0 ? sms : 148;
+  c->cluster = choose_cluster(N, c->num_sms);
   float* om = static_cast<float*>(malloc(sizeof(float) * N));
   if (!om) { free(c); return REGTOPK_ERR_INVALID_ARG; }
   for (int n = 0; n < N; ++n) om[n] = params->omega ? params->omega[n] : 1.0f / (float)N;
@@ -1075,9 +1212,9 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
 
   SampleArgs sa;
   sa.grads = grads; sa.grad_ld = grad_ld; sa.eps = at<float>(c, L.off_eps); sa.ld = L.ld; sa.d = c->d;
+  sa.k = c->k;
   sa.k_target = use_marks ? (2 * c->k < c->d ? 2 * c->k : c->d) : c->k;
   sa.ctl = at<WorkerCtl>(c, L.off_ctl); sa.gctl = at<GlobalCtl>(c, L.off_gctl);
-  sa.tcount = at<u32>(c, L.off_tcount); sa.ntiles = L.ntiles;
   sa.force_dense = (c->flags & REGTOPK_FLAG_FORCE_DENSE_SELECT) ? 1 : 0;
   if (bf16) k_sample_cutoff<true><<<c->N, kBlockSel, sample_smem(), c->stream>>>(sa);
   else k_sample_cutoff<false><<<c->N, kBlockSel, sample_smem(), c->stream>>>(sa);
@@ -1085,7 +1222,7 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
 
   StreamArgs st;
   st.grads = grads; st.grad_ld = grad_ld; st.eps = at<float>(c, L.off_eps); st.ld = L.ld; st.d = c->d;
-  st.N = c->N; st.ctl = sa.ctl; st.cand = at<u64>(c, L.off_candA); st.cap = L.capA; st.stride = L.capB;
+  st.N = c->N; st.ctl = sa.ctl; st.cand = at<u64>(c, L.off_candA); st.cap = L.capA; st.stride = L.stride;
   const bool prof = c->profiling && c->n_events < kMaxProfile;
   if (prof) cudaEventRecord(c->ev0[c->n_events], c->stream);
   if (bf16) { if (vec) launch_stream<true, true>(c, st, 3); else launch_stream<true, false>(c, st, 2); }
@@ -1093,44 +1230,24 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   if (prof) cudaEventRecord(c->ev1[c->n_events++], c->stream);
   if ((rc = after_launch(c))) return rc;
 
-  if (use_marks) {
-    OverrideArgs oa;
-    oa.eps = at<float>(c, L.off_eps); oa.ld = L.ld; oa.g_prev = at<float>(c, L.off_g);
-    oa.prev_idx = at<int32_t>(c, L.off_idx[prev]); oa.prev_val = at<float>(c, L.off_val[prev]);
-    oa.omega = at<float>(c, L.off_omega); oa.mu = c->mu; oa.k = c->k; oa.N = c->N; oa.ctl = sa.ctl;
-    oa.ovr_key = at<u32>(c, L.off_ovr_key); oa.ovr_comp = at<u64>(c, L.off_ovr_comp);
-    const int64_t total = c->k * c->N;
-    int64_t blocks = (total + 255) / 256;
-    if (blocks > (int64_t)c->num_sms * 16) blocks = (int64_t)c->num_sms * 16;
-    k_override<<<(unsigned)blocks, 256, 0, c->stream>>>(oa);
-    if ((rc = after_launch(c))) return rc;
-  }
-
-  SelectArgs se;
-  se.ctl = sa.ctl; se.gctl = sa.gctl; se.candA = at<u64>(c, L.off_candA); se.capA = L.capA;
-  se.candB = at<u64>(c, L.off_candB); se.stride = L.capB; se.ovr_comp = at<u64>(c, L.off_ovr_comp);
-  se.prev_idx = at<int32_t>(c, L.off_idx[prev]); se.bitmask = at<u32>(c, L.off_mask); se.W = L.W;
-  se.tcount = sa.tcount; se.toff = at<u32>(c, L.off_toff); se.ntiles = L.ntiles; se.k = c->k;
-  se.use_marks = use_marks; se.has_prev = has_prev; se.phase = 0;
-  k_select<<<c->N, kBlockSel, 0, c->stream>>>(se);
-  if ((rc = after_launch(c))) return rc;
-
-  DenseArgs da;
-  da.ctl = sa.ctl; da.gctl = sa.gctl; da.eps = at<float>(c, L.off_eps); da.ld = L.ld; da.d = c->d;
-  da.k = c->k; da.bitmask = at<u32>(c, L.off_mask); da.W = L.W; da.prev_idx = se.prev_idx;
-  da.ovr_key = at<u32>(c, L.off_ovr_key); da.candA = se.candA; da.stride = L.capB; da.use_marks = use_marks;
-  k_dense_select<<<c->N, kBlockSel, 0, c->stream>>>(da);
-  if ((rc = after_launch(c))) return rc;
-  se.phase = 1;
-  k_select<<<c->N, kBlockSel, 0, c->stream>>>(se);
-  if ((rc = after_launch(c))) return rc;
-
-  EmitArgs em;
-  em.bitmask = se.bitmask; em.W = L.W; em.tcount = se.tcount; em.toff = se.toff; em.ntiles = L.ntiles;
-  em.eps = at<float>(c, L.off_eps); em.ld = L.ld; em.k = c->k; em.out_idx = out_idx; em.out_val = out_val;
-  em.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); em.cur_val = at<float>(c, L.off_val[c->cur]);
-  k_emit<<<dim3((unsigned)L.ntiles, (unsigned)c->N), 256, 0, c->stream>>>(em);
-  if ((rc = after_launch(c))) return rc;
+  PostArgs pa;
+  pa.ctl = sa.ctl; pa.gctl = sa.gctl; pa.eps = at<float>(c, L.off_eps); pa.ld = L.ld; pa.d = c->d; pa.k = c->k;
+  pa.g_prev = at<float>(c, L.off_g);
+  pa.prev_idx = at<int32_t>(c, L.off_idx[prev]); pa.prev_val = at<float>(c, L.off_val[prev]);
+  pa.omega = at<float>(c, L.off_omega); pa.mu = c->mu;
+  pa.ovr_key = at<u32>(c, L.off_ovr_key); pa.ovr_comp = at<u64>(c, L.off_ovr_comp);
+  pa.candA = at<u64>(c, L.off_candA); pa.candB = at<u64>(c, L.off_candB); pa.capA = L.capA; pa.stride = L.stride;
+  pa.bitmask = at<u32>(c, L.off_mask); pa.wprefix = at<u32>(c, L.off_wprefix); pa.W = L.W;
+  pa.out_idx = out_idx; pa.out_val = out_val;
+  pa.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); pa.cur_val = at<float>(c, L.off_val[c->cur]);
+  pa.use_marks = use_marks; pa.has_prev = has_prev;
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  post_config(&cfg, attr, c->N, c->cluster, c->stream);
+  cudaError_t le = cudaLaunchKernelEx(&cfg, k_post, pa);
+  c->launches++;
+  if (le != cudaSuccess) return note_cuda(c, le);
+  if ((rc = note_cuda(c, cudaGetLastError()))) return rc;
 
   c->stepped = 1;
   return REGTOPK_OK;
@@ -1141,14 +1258,16 @@ int regtopk_aggregate(regtopk_ctx* c, float* out_g) {
   if (!c->stepped) return REGTOPK_ERR_SEQUENCE;
   const Layout& L = c->L;
   AggArgs a;
-  a.g = at<float>(c, L.off_g); a.d = c->d; a.N = c->N; a.k = c->k;
+  a.g = at<float>(c, L.off_g); a.N = c->N; a.k = c->k;
   a.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); a.cur_val = at<float>(c, L.off_val[c->cur]);
-  a.prev_idx = at<int32_t>(c, L.off_idx[c->cur ^ 1]); a.omega = at<float>(c, L.off_omega);
+  a.prev_idx = at<int32_t>(c, L.off_idx[c->cur ^ 1]);
+  a.bitmask = at<u32>(c, L.off_mask); a.wprefix = at<u32>(c, L.off_wprefix); a.W = L.W;
+  a.omega = at<float>(c, L.off_omega);
   a.has_prev = c->round >= 1;
-  int64_t blocks = (int64_t)c->num_sms * 8;
-  if (blocks > c->d) blocks = c->d;
-  const size_t smem = (size_t)4 * c->N * sizeof(int64_t);
-  k_aggregate<<<(unsigned)blocks, 256, smem, c->stream>>>(a);
+  const int64_t threads = (a.has_prev ? 2 : 1) * c->k * (int64_t)c->N;
+  int64_t blocks = (threads + 255) / 256;
+  if (blocks > (int64_t)c->num_sms * 32) blocks = (int64_t)c->num_sms * 32;
+  k_aggregate<<<(unsigned)blocks, 256, 0, c->stream>>>(a);
   int rc = after_launch(c);
   if (rc) return rc;
   if (out_g)
