@@ -15,7 +15,7 @@
 //                     zeroing the residual there.  If the cutoff guess was too high or the list
 //                     overflowed, the same cluster runs an exact radix select over the whole row.
 //   k_aggregate       server sum in worker order, one thread per sent pair, ranks looked up through
-//                     the per-word prefix counts written during emission
+//                     the per-unit prefix counts written during emission
 //
 // The selection key of an entry is the bit pattern of its non-negative binary32 score, which orders
 // like the score; the 64-bit composite (key << 32 | ~index) orders like (score descending, index
@@ -209,6 +209,7 @@ struct SampleArgs {
   int64_t k_target;  // entries the cutoff should leave above it (k, or 2k when overrides can demote)
   WorkerCtl* ctl;
   GlobalCtl* gctl;
+  u32* ghist;  // [N][4][kBins], cleared here for k_post
   int force_dense;
 };
 
@@ -223,6 +224,7 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
   const int tid = threadIdx.x;
   WorkerCtl* ctl = p.ctl + n;
 
+  for (int i = tid; i < 4 * kBins; i += blockDim.x) p.ghist[(size_t)n * 4 * kBins + i] = 0;
   if (p.force_dense) {
     if (tid == 0) {
       ctl->cutoff = kFull;  // no key reaches it: the stream pass collects nothing
@@ -442,98 +444,20 @@ __global__ void __launch_bounds__(kStreamThreads) k_stream(StreamArgs p) {
 
 
 // ---------------------------------------------------------------------------------------------
-// cluster-wide helpers (every block of the cluster calls them, the same number of times)
+// k_post: one thread-block cluster per worker.  The cluster's blocks meet only at the hardware
+// cluster barrier; what they exchange (histograms, list lengths, per-block totals) goes through
+// global memory, which the barrier's release/acquire makes visible.  Every block of a cluster
+// reaches every barrier: all branches that contain one depend only on values that are the same in
+// all blocks of the cluster.
 // ---------------------------------------------------------------------------------------------
 struct PostShared {
-  u32 hist[kBins];     // this block's histogram; peers read it through distributed shared memory
-  u32 merged[kBins];   // this block's slice of the cluster-wide histogram
-  u32 tot[kMaxCluster];
-  u32 xch[kMaxCluster];
-  u32 res[2];
+  u32 hist[kBins];    // histogram of this block, then of the cluster
+  u32 spare[kBins];   // with hist: 8192 words reused as item storage and per-warp emission lists
   u32 fres[3];
   u32 scan[33];
   u32 cnt;
 };
 
-struct FindResult {
-  u32 bin, above, total;
-};
-
-// The blocks of a cluster have each filled sh.hist (kBins bins).  Returns, in every block, the bin of
-// the merged histogram that holds the r-th entry counted from the top, the entries above it, and the
-// grand total; bin == kFull if the total is below r.  Three cluster barriers.
-__device__ FindResult cluster_find_from_top(cg::cluster_group& cl, PostShared& sh, u32 r) {
-  const u32 CS = cl.num_blocks(), rk = cl.block_rank();
-  const int per = kBins / (int)CS;
-  const int tid = threadIdx.x;
-  cl.sync();  // all local histograms complete
-  u32 part = 0;
-  for (int b = tid; b < per; b += blockDim.x) {
-    const int bin = (int)rk * per + b;
-    u32 sum = 0;
-    for (u32 c = 0; c < CS; ++c) sum += cl.map_shared_rank(sh.hist, c)[bin];
-    sh.merged[b] = sum;
-    part += sum;
-  }
-  u32 slice_total;
-  block_excl_scan(part, sh.scan, &slice_total);
-  if (tid < (int)CS) cl.map_shared_rank(sh.tot, tid)[rk] = slice_total;
-  if (tid == 0) sh.res[0] = kFull;
-  cl.sync();  // slice totals delivered; every peer has finished reading this block's histogram
-  u32 acc = 0, total = 0;
-  int q = -1;
-  for (int s = (int)CS - 1; s >= 0; --s) {
-    const u32 t = sh.tot[s];
-    if (q < 0 && acc + t >= r) q = s;
-    if (q < 0) acc += t;
-    total += t;
-  }
-  if (q == (int)rk) {  // block-uniform
-    block_find_from_top(sh.merged, per, r - acc, sh.scan, sh.fres);
-    if (tid < (int)CS) {
-      u32* dst = cl.map_shared_rank(sh.res, tid);
-      dst[0] = sh.fres[0] == kFull ? kFull : (u32)((int)rk * per) + sh.fres[0];
-      dst[1] = acc + sh.fres[1];
-    }
-  }
-  cl.sync();  // result delivered
-  FindResult out;
-  out.bin = sh.res[0];
-  out.above = sh.res[1];
-  out.total = total;
-  return out;
-}
-
-// Exclusive prefix of one value per block over the cluster's block ranks, and the total.  Two barriers.
-__device__ u32 cluster_excl_sum(cg::cluster_group& cl, PostShared& sh, u32 v, u32* total) {
-  const u32 CS = cl.num_blocks(), rk = cl.block_rank();
-  if (threadIdx.x < CS) cl.map_shared_rank(sh.xch, threadIdx.x)[rk] = v;
-  cl.sync();
-  u32 pre = 0, tot = 0;
-  for (u32 c = 0; c < CS; ++c) {
-    const u32 t = sh.xch[c];
-    if (c < rk) pre += t;
-    tot += t;
-  }
-  *total = tot;
-  cl.sync();  // everyone has read; the exchange array may be written again
-  return pre;
-}
-
-__device__ __forceinline__ u32 warp_reserve_global(bool pred, u32* counter) {
-  const u32 m = __ballot_sync(kFull, pred);
-  if (m == 0) return 0;
-  const int lane = threadIdx.x & 31;
-  const int leader = __ffs(m) - 1;
-  u32 base = 0;
-  if (lane == leader) base = atomicAdd(counter, (u32)__popc(m));
-  base = __shfl_sync(kFull, base, leader);
-  return base + (u32)__popc(m & ((1u << lane) - 1u));
-}
-
-// ---------------------------------------------------------------------------------------------
-// k_post: one cluster per worker.
-// ---------------------------------------------------------------------------------------------
 struct PostArgs {
   WorkerCtl* ctl;
   GlobalCtl* gctl;
@@ -552,16 +476,30 @@ struct PostArgs {
   u64* candB;     // [N][stride]
   int64_t capA;
   int64_t stride;  // capA + k: what one histogram bin can hold (all candidates plus all overrides)
-  u32* bitmask;    // [N][W] winners of this round (last round's on entry)
-  u32* wprefix;    // [N][W] winners before each non-empty mask word (rank directory for k_aggregate)
+  u32* ghist;      // [N][4][kBins] cluster-wide histograms, zeroed by k_sample_cutoff
+  u32* btot;       // [N][2][kMaxCluster] per-block totals
+  const u32* mask_old;  // [N][W] last round's mask (marks the previous support)
+  u32* mask_new;   // [N][W] this round's mask; on entry it holds the mask of two rounds ago
+  u32* uprefix;    // [N][W/8] winners before each 8-word unit of the mask (rank directory for k_aggregate)
   int64_t W;       // words per row, a multiple of 32
   int32_t* out_idx;
   float* out_val;
-  int32_t* cur_idx;
+  int32_t* cur_idx;  // on entry: the pairs of two rounds ago (the bits to clear in mask_new)
   float* cur_val;
   int use_marks;  // previous support carries regularised scores (round >= 1, mu > 0)
-  int has_prev;   // the bitmask holds last round's mask, to be cleared
+  int has_stale;  // mask_new holds an old mask (round >= 2)
 };
+
+__device__ __forceinline__ u32 warp_reserve_global(bool pred, u32* counter) {
+  const u32 m = __ballot_sync(kFull, pred);
+  if (m == 0) return 0;
+  const int lane = threadIdx.x & 31;
+  const int leader = __ffs(m) - 1;
+  u32 base = 0;
+  if (lane == leader) base = atomicAdd(counter, (u32)__popc(m));
+  base = __shfl_sync(kFull, base, leader);
+  return base + (u32)__popc(m & ((1u << lane) - 1u));
+}
 
 __device__ __forceinline__ void set_winner(u32* mask, u32 idx) {
   atomicOr(&mask[idx >> 5], 1u << (idx & 31));
@@ -572,10 +510,31 @@ __device__ __forceinline__ u32 select_bin(u32 key, u32 cutoff, u32 shift) {
   return b < (u32)(kBins - 1) ? b : (u32)(kBins - 1);
 }
 
+// Add this block's histogram to the cluster's in global memory (non-empty bins only).
+__device__ __forceinline__ void flush_hist(const u32* s_hist, u32* g_hist) {
+  for (int i = threadIdx.x; i < kBins; i += blockDim.x) {
+    const u32 v = s_hist[i];
+    if (v) atomicAdd(&g_hist[i], v);
+  }
+}
+
+// After the cluster barrier: every block loads the cluster's histogram and finds the bin of the
+// r-th entry from the top by itself (all blocks get the same answer).
+__device__ __forceinline__ void load_and_find(PostShared& sh, const u32* g_hist, u32 r, u32* bin,
+                                              u32* above, u32* total) {
+  for (int i = threadIdx.x; i < kBins; i += blockDim.x) sh.hist[i] = __ldcg(&g_hist[i]);
+  __syncthreads();
+  block_find_from_top(sh.hist, kBins, r, sh.scan, sh.fres);
+  *bin = sh.fres[0];
+  *above = sh.fres[1];
+  *total = sh.fres[2];
+  __syncthreads();
+}
+
 // Score key of entry j for the dense path: the override's on the previous support, bits(|a|) elsewhere.
 __device__ __forceinline__ u32 dense_key(const PostArgs& p, int n, int64_t j) {
   if (p.use_marks) {
-    const u32 w = p.bitmask[(size_t)n * p.W + (j >> 5)];
+    const u32 w = p.mask_old[(size_t)n * p.W + (j >> 5)];
     if ((w >> (j & 31)) & 1u) {
       const int32_t* pi = p.prev_idx + (size_t)n * p.k;
       int64_t lo = 0, hi = p.k;
@@ -583,47 +542,51 @@ __device__ __forceinline__ u32 dense_key(const PostArgs& p, int n, int64_t j) {
         const int64_t mid = (lo + hi) >> 1;
         if (pi[mid] < (int32_t)j) lo = mid + 1; else hi = mid;
       }
-      return p.ovr_key[(size_t)n * p.k + lo];
+      return __ldcg(&p.ovr_key[(size_t)n * p.k + lo]);
     }
   }
   return __float_as_uint(p.eps[(size_t)n * p.ld + j]) & 0x7FFFFFFFu;
 }
 
-// Leader block only: pick the `need` largest composites of list[0..count) and set them as winners.
-// Uses `other` (same capacity) as the second buffer of the radix passes.
-__device__ void refine_list(PostShared& sh, u32* mask, GlobalCtl* gctl, u64* list, u64* other,
-                            u32 count, u32 need) {
+// One block: among list[0..count) (count <= 1024, unique composites) set the `need` largest as
+// winners, but only those whose mask word lies in [w0, w1) (the caller's share of the mask).
+__device__ void refine_small(PostShared& sh, u32* mask, const u64* list, u32 count, u32 need,
+                             int64_t w0, int64_t w1) {
+  u64* s_items = reinterpret_cast<u64*>(sh.hist);
   const int tid = threadIdx.x;
-  if (need == 0) return;
-  if (need >= count) {
-    for (u32 i = tid; i < count; i += blockDim.x) set_winner(mask, composite_idx(list[i]));
-    return;
+  u64 mine = 0ull;
+  if ((u32)tid < count) {
+    mine = __ldcg(&list[tid]);
+    s_items[tid] = mine;
   }
-  if (count <= (u32)kBins) {
-    // small list: rank every item by counting the items above it (composites are unique)
-    u64* s_items = reinterpret_cast<u64*>(sh.hist);  // hist and merged are contiguous: kBins u64
-    for (u32 i = tid; i < count; i += blockDim.x) s_items[i] = list[i];
-    __syncthreads();
-    for (u32 i = tid; i < count; i += blockDim.x) {
-      const u64 c = s_items[i];
+  __syncthreads();
+  if ((u32)tid < count) {
+    const u32 idx = composite_idx(mine);
+    const int64_t wi = (int64_t)(idx >> 5);
+    if (wi >= w0 && wi < w1) {
       u32 above = 0;
-      for (u32 j = 0; j < count; ++j) above += s_items[j] > c ? 1u : 0u;
-      if (above < need) set_winner(mask, composite_idx(c));
+      for (u32 j = 0; j < count; ++j) above += s_items[j] > mine ? 1u : 0u;
+      if (above < need) set_winner(mask, idx);
     }
-    __syncthreads();
-    return;
   }
-  // general case (long runs of equal keys): radix passes over all 64 composite bits
+  __syncthreads();
+}
+
+// Leader block only: the `need` largest composites of list[0..count), any count, by radix passes
+// over all 64 bits.  `other` (same capacity) is the second buffer.
+__device__ void refine_large(PostShared& sh, u32* mask, GlobalCtl* gctl, u64* list, u64* other,
+                             u32 count, u32 need) {
+  const int tid = threadIdx.x;
   u64* src = list;
   u64* dst = other;
   u32 nsrc = count;
   for (int shift = 56; shift >= 0; shift -= 8) {
     if (need == 0) return;
-    if (need == nsrc) break;
+    if (need >= nsrc) break;
     for (int i = tid; i < 256; i += blockDim.x) sh.hist[i] = 0;
     if (tid == 0) sh.cnt = 0;
     __syncthreads();
-    for (u32 i = tid; i < nsrc; i += blockDim.x) atomicAdd(&sh.hist[(u32)(src[i] >> shift) & 255u], 1u);
+    for (u32 i = tid; i < nsrc; i += blockDim.x) atomicAdd(&sh.hist[(u32)(__ldcg(&src[i]) >> shift) & 255u], 1u);
     __syncthreads();
     block_find_from_top(sh.hist, 256, need, sh.scan, sh.fres);
     const u32 b = sh.fres[0], above = sh.fres[1];
@@ -638,7 +601,7 @@ __device__ void refine_list(PostShared& sh, u32* mask, GlobalCtl* gctl, u64* lis
       u64 c = 0ull;
       u32 dg = 0;
       if (i < nsrc) {
-        c = src[i];
+        c = __ldcg(&src[i]);
         dg = (u32)(c >> shift) & 255u;
         if (dg > b) set_winner(mask, composite_idx(c));
       }
@@ -652,11 +615,48 @@ __device__ void refine_list(PostShared& sh, u32* mask, GlobalCtl* gctl, u64* lis
     __syncthreads();
     u64* t = src; src = dst; dst = t;
   }
-  if (need == nsrc) {
-    for (u32 i = tid; i < nsrc; i += blockDim.x) set_winner(mask, composite_idx(src[i]));
+  if (need >= nsrc) {
+    for (u32 i = tid; i < nsrc; i += blockDim.x) set_winner(mask, composite_idx(__ldcg(&src[i])));
   } else if (need != 0) {
     if (tid == 0) atomicOr(&gctl->err, kErrRefine);  // all bits consumed: composites were not unique
   }
+}
+
+constexpr int kEmitUnits = 2 * kBins;  // 8-word units per emission chunk (the shared prefix array holds one word each)
+
+// Count the winners of the units [cu0, min(cu0 + kEmitUnits, bu1)) of a mask row: s_up[u] receives
+// the winners before unit u within the chunk; returns the chunk's total.  A thread owns 8 consecutive
+// units.  Every thread of the block must call it.
+__device__ u32 emit_count_chunk(PostShared& sh, const u32* mask, int64_t cu0, int64_t bu1, u32* s_up) {
+  const int tid = threadIdx.x;
+  u32 c[8];
+  u32 sum = 0;
+  uint4 x[8], y[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int64_t u = cu0 + tid * 8 + i;
+    x[i] = make_uint4(0, 0, 0, 0);
+    y[i] = x[i];
+    if (u < bu1) {
+      x[i] = __ldcg(reinterpret_cast<const uint4*>(mask + u * 8));
+      y[i] = __ldcg(reinterpret_cast<const uint4*>(mask + u * 8 + 4));
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    c[i] = __popc(x[i].x) + __popc(x[i].y) + __popc(x[i].z) + __popc(x[i].w) + __popc(y[i].x) +
+           __popc(y[i].y) + __popc(y[i].z) + __popc(y[i].w);
+    sum += c[i];
+  }
+  u32 total;
+  u32 run = block_excl_scan(sum, sh.scan, &total);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    s_up[tid * 8 + i] = run;
+    run += c[i];
+  }
+  __syncthreads();
+  return total;
 }
 
 __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
@@ -664,13 +664,13 @@ __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
   cg::cluster_group cl = cg::this_cluster();
   const u32 CS = cl.num_blocks(), rk = cl.block_rank();
   const int n = blockIdx.x / CS;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
   const u32 stride_t = CS * blockDim.x;        // threads of the cluster
   const u32 first_t = rk * blockDim.x + tid;   // this thread's index among them
   WorkerCtl* ctl = p.ctl + n;
   const u32 cutoff = ctl->cutoff, bshift = ctl->bin_shift;
   const u32 cand_count = ctl->cand_count;
-  bool dense = ctl->force_dense != 0;          // identical in every block: nothing writes it here
+  bool dense = ctl->force_dense != 0;          // the same in every block: nothing writes it here
   const u32 k = (u32)p.k;
   u64* A = p.candA + (size_t)n * p.stride;
   u64* B = p.candB + (size_t)n * p.stride;
@@ -678,81 +678,103 @@ __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
   u32* okey = p.ovr_key + (size_t)n * p.k;
   const int32_t* prev_idx = p.prev_idx + (size_t)n * p.k;
   const float* prev_val = p.prev_val + (size_t)n * p.k;
-  u32* mask = p.bitmask + (size_t)n * p.W;
-  u32* wpre = p.wprefix + (size_t)n * p.W;
+  const u32* mask_old = p.mask_old + (size_t)n * p.W;
+  u32* mask = p.mask_new + (size_t)n * p.W;
+  u32* ghist = p.ghist + (size_t)n * 4 * kBins;
+  u32* btot = p.btot + (size_t)n * 2 * kMaxCluster;
   float* eps_row = p.eps + (size_t)n * p.ld;
+  const size_t obase = (size_t)n * p.k;
   const bool overflow = (u64)cand_count > (u64)p.capA;
   const u32 ncand = overflow ? (u32)p.capA : cand_count;
   const u32 novr = p.use_marks ? k : 0u;
+  // this block's share of the mask for the emission: units of 8 words
+  const int64_t U = p.W >> 3;
+  const int64_t bu0 = (int64_t)(((u64)rk * (u64)U) / CS), bu1 = (int64_t)(((u64)(rk + 1) * (u64)U) / CS);
 
-  // ---- regularised scores on the previous support (Eq. (Delta_def), Algorithm 2 step 9) ----
-  if (p.use_marks) {
-    const float w = p.omega[n];
-    for (u32 i = first_t; i < k; i += stride_t) {
-      const int32_t j = prev_idx[i];
-      const float a = eps_row[j];
-      const float num = __fsub_rn(p.g_prev[j], __fmul_rn(w, prev_val[i]));
-      const float den = __fmul_rn(w, a);
-      float m = 1.0f;
-      if (den != 0.0f) {
-        const float delta = __fdiv_rn(num, den);
-        const float r = fabsf(__fadd_rn(1.0f, delta));
-        m = tanh_fixed(__fdiv_rn(r, p.mu));
-      }
-      const u32 key = __float_as_uint(__fmul_rn(fabsf(a), m));
-      okey[i] = key;
-      O[i] = key >= cutoff ? make_composite(key, (u32)j) : 0ull;
-    }
-  }
   for (int i = tid; i < kBins; i += blockDim.x) sh.hist[i] = 0;
-  cl.sync();  // override keys visible to the whole cluster; histograms cleared
-
-  FindResult fr;
-  fr.bin = kFull; fr.above = 0; fr.total = 0;
-  if (!dense) {
-    // ---- filter and histogram: candidates on the previous support are dropped (their score is the
-    //      override's); every thread keeps the same items in the later classify pass ----
-    for (u32 i = first_t; i < ncand; i += stride_t) {
-      const u64 c = A[i];
-      if (p.use_marks) {
-        const u32 idx = composite_idx(c);
-        if ((mask[idx >> 5] >> (idx & 31)) & 1u) {
-          A[i] = 0ull;
-          continue;
+  __syncthreads();
+  // ---- one fused sweep, so that the independent loads of its three jobs are in flight together:
+  //   (a) the mask buffer of this round still holds the mask of two rounds ago: clear those words;
+  //   (b) regularised scores on the previous support (Eq. (Delta_def), Algorithm 2 step 9);
+  //   (c) filter and histogram the candidates: those on the previous support are dropped (their
+  //       score is the override's); a thread meets the same items again in the classify pass ----
+  {
+    const float w = p.omega[n];
+    const u32 span = !dense && ncand > k ? ncand : k;
+    for (u32 i = first_t; i < span; i += stride_t) {
+      const bool in_k = i < k;
+      const bool do_ovr = in_k && p.use_marks;
+      const bool do_cand = !dense && i < ncand;
+      // first wave of loads
+      const int32_t stale = (in_k && p.has_stale) ? p.cur_idx[obase + i] : 0;
+      const int32_t j = do_ovr ? prev_idx[i] : 0;
+      const float ap = do_ovr ? prev_val[i] : 0.0f;
+      const u64 c = do_cand ? A[i] : 0ull;
+      // second wave, dependent on the first
+      const float a = do_ovr ? eps_row[j] : 0.0f;
+      const float G = do_ovr ? p.g_prev[j] : 0.0f;
+      const u32 cidx = composite_idx(c);
+      const u32 mword = (do_cand && p.use_marks) ? mask_old[cidx >> 5] : 0u;
+      if (in_k && p.has_stale) mask[(u32)stale >> 5] = 0u;
+      if (do_ovr) {
+        const float num = __fsub_rn(G, __fmul_rn(w, ap));
+        const float den = __fmul_rn(w, a);
+        float m = 1.0f;
+        if (den != 0.0f) {
+          const float delta = __fdiv_rn(num, den);
+          const float r = fabsf(__fadd_rn(1.0f, delta));
+          m = tanh_fixed(__fdiv_rn(r, p.mu));
         }
+        const u32 key = __float_as_uint(__fmul_rn(fabsf(a), m));
+        const u64 oc = key >= cutoff ? make_composite(key, (u32)j) : 0ull;
+        okey[i] = key;
+        O[i] = oc;
+        if (!dense && oc) atomicAdd(&sh.hist[select_bin(key, cutoff, bshift)], 1u);
       }
-      atomicAdd(&sh.hist[select_bin((u32)(c >> 32), cutoff, bshift)], 1u);
+      if (do_cand) {
+        if ((mword >> (cidx & 31)) & 1u) A[i] = 0ull;
+        else atomicAdd(&sh.hist[select_bin((u32)(c >> 32), cutoff, bshift)], 1u);
+      }
     }
-    for (u32 i = first_t; i < novr; i += stride_t) {
-      const u64 c = O[i];
-      if (c) atomicAdd(&sh.hist[select_bin((u32)(c >> 32), cutoff, bshift)], 1u);
-    }
-    fr = cluster_find_from_top(cl, sh, k);
-    if (fr.bin == kFull || overflow) dense = true;  // cutoff guessed too high, or the list overflowed
-    if (rk == 0 && tid == 0) ctl->n_valid = fr.total;
+  }
+  __syncthreads();
+  if (!dense) flush_hist(sh.hist, ghist);
+  cl.sync();  // (1) cluster histogram complete; stale mask words cleared; override keys written
+
+  u32 b1 = kFull, above1 = 0, nvalid = 0;
+  if (!dense) {
+    load_and_find(sh, ghist, k, &b1, &above1, &nvalid);
+    if (b1 == kFull || overflow) dense = true;  // cutoff guessed too high, or the list overflowed
+    if (rk == 0 && tid == 0) ctl->n_valid = nvalid;
   }
 
   if (!dense) {
-    // every probe of the old mask is done: clear it (whole words; all their bits are old marks)
-    if (p.has_prev)
-      for (u32 i = first_t; i < k; i += stride_t) mask[(u32)prev_idx[i] >> 5] = 0u;
-    cl.sync();
     // ---- classify: above the bin -> winner; inside it -> refinement list ----
-    const u32 total_items = ncand + novr;
-    const u32 iters = (total_items + stride_t - 1) / stride_t;
-    for (u32 it = 0; it < iters; ++it) {
-      const u32 i = it * stride_t + first_t;
-      u64 c = 0ull;
-      if (i < ncand) c = A[i];
-      else if (i < total_items) c = O[i - ncand];
-      const u32 bin = c ? select_bin((u32)(c >> 32), cutoff, bshift) : 0u;
-      if (c && bin > fr.bin) set_winner(mask, composite_idx(c));
-      const bool inbin = c && bin == fr.bin;
-      const u32 pos = warp_reserve_global(inbin, &ctl->bcount);
-      if (inbin) B[pos] = c;
+    // (each thread re-reads exactly the list slots it wrote or filtered before the barrier)
+    for (int part = 0; part < 2; ++part) {
+      const u64* items = part == 0 ? A : O;
+      const u32 count = part == 0 ? ncand : novr;
+      const u32 iters = (count + stride_t - 1) / stride_t;
+      for (u32 it = 0; it < iters; ++it) {
+        const u32 i = it * stride_t + first_t;
+        const u64 c = i < count ? items[i] : 0ull;
+        const u32 bin = c ? select_bin((u32)(c >> 32), cutoff, bshift) : 0u;
+        if (c && bin > b1) set_winner(mask, composite_idx(c));
+        const bool inbin = c && bin == b1;
+        const u32 pos = warp_reserve_global(inbin, &ctl->bcount);
+        if (inbin) B[pos] = c;
+      }
     }
-    cl.sync();
-    if (rk == 0) refine_list(sh, mask, p.gctl, B, A, __ldcg(&ctl->bcount), k - fr.above);
+    cl.sync();  // (2) refinement list complete
+    const u32 nB = __ldcg(&ctl->bcount);
+    const u32 need = k - above1;
+    if (nB <= 1024u) {
+      // every block ranks the short list itself and sets the winners of its own share of the mask
+      refine_small(sh, mask, B, nB, need, bu0 * 8, bu1 * 8);
+    } else {
+      if (rk == 0) refine_large(sh, mask, p.gctl, B, A, nB, need);
+      cl.sync();  // (2b) the leader's winners are set
+    }
   } else {
     // ---- exact selection over the whole row: three radix digits of the 31-bit key ----
     if (rk == 0 && tid == 0) atomicAdd(&p.gctl->dense_workers, 1ull);
@@ -772,10 +794,13 @@ __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
         const u32 key = dense_key(p, n, j);
         if (lv == 0 || (key >> (shf + widths[lv])) == prefix) atomicAdd(&sh.hist[(key >> shf) & nbm], 1u);
       }
-      const FindResult r = cluster_find_from_top(cl, sh, need);
-      if (r.bin == kFull) bad = true;
-      const u32 b = r.bin == kFull ? 0u : r.bin;
-      need -= r.bin == kFull ? 0u : r.above;
+      __syncthreads();
+      flush_hist(sh.hist, ghist + (1 + lv) * kBins);
+      cl.sync();
+      u32 b, above, total;
+      load_and_find(sh, ghist + (1 + lv) * kBins, need, &b, &above, &total);
+      if (b == kFull) { bad = true; b = 0; above = 0; }
+      need -= above;
       prefix = (prefix << widths[lv]) | b;
     }
     const u32 T = prefix;          // key of the k-th largest score
@@ -796,8 +821,14 @@ __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
     }
     u32 block_ties;
     block_excl_scan(my_ties, sh.scan, &block_ties);
-    u32 all_ties;
-    u32 taken = cluster_excl_sum(cl, sh, block_ties, &all_ties);  // ties in lower-index blocks
+    if (tid == 0) btot[kMaxCluster + rk] = block_ties;
+    cl.sync();
+    u32 taken = 0, all_ties = 0;  // ties in lower-index blocks, and in the whole row
+    for (u32 c = 0; c < CS; ++c) {
+      const u32 t = __ldcg(&btot[kMaxCluster + c]);
+      if (c < rk) taken += t;
+      all_ties += t;
+    }
     if (all_ties < need) bad = true;
     // ties in index order: the first `need` of them
     for (int64_t base = c0; base < c1 && taken < need; base += blockDim.x) {
@@ -808,92 +839,103 @@ __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
       if (tie && rank < need) A[n_gt + rank] = make_composite(T, (u32)j);
       taken += total;
     }
-    cl.sync();  // winner list complete; nobody reads the old mask any more
+    cl.sync();  // winner list complete
     if (rk == 0 && tid == 0 && (bad || __ldcg(&ctl->acount) != n_gt)) atomicOr(&p.gctl->err, kErrDenseSelect);
-    if (p.has_prev)
-      for (u32 i = first_t; i < k; i += stride_t) mask[(u32)prev_idx[i] >> 5] = 0u;
-    cl.sync();
     if (!bad)
       for (u32 i = first_t; i < k; i += stride_t) set_winner(mask, composite_idx(__ldcg(&A[i])));
+    cl.sync();  // every winner bit is set
   }
-  cl.sync();  // every winner bit is set
 
-  // ---- emission: ordered walk of the bitmask; blocks and warps own contiguous ranges of 32-word groups ----
-  const int64_t G = p.W >> 5;
-  const int64_t g0 = (int64_t)(((u64)rk * (u64)G) / CS), g1 = (int64_t)(((u64)(rk + 1) * (u64)G) / CS);
-  const int nw = blockDim.x >> 5;
-  const int64_t wg0 = g0 + ((g1 - g0) * warp) / nw, wg1 = g0 + ((g1 - g0) * (warp + 1)) / nw;
-  u32 wsum = 0;
-  for (int64_t g = wg0; g < wg1; ++g) wsum += __popc(__ldcg(&mask[g * 32 + lane]));
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(kFull, wsum, o);
-  u32 block_total;
-  u32 warp_pre = block_excl_scan(lane == 0 ? wsum : 0u, sh.scan, &block_total);
-  warp_pre = __shfl_sync(kFull, warp_pre, 0);
-  u32 all_total;
-  const u32 block_pre = cluster_excl_sum(cl, sh, block_total, &all_total);
-  if (rk == 0 && tid == 0 && all_total != k) atomicOr(&p.gctl->err, kErrCountMismatch);
-  if (all_total == k) {
-    u32 running = block_pre + warp_pre;
-    const size_t obase = (size_t)n * p.k;
-    for (int64_t g = wg0; g < wg1; ++g) {
-      const u32 word = __ldcg(&mask[g * 32 + lane]);
-      const u32 c = __popc(word);
-      u32 inc = c;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const u32 t = __shfl_up_sync(kFull, inc, o);
-        if (lane >= o) inc += t;
-      }
-      const u32 T = __shfl_sync(kFull, inc, 31);
-      if (T == 0) continue;
-      const u32 pre = inc - c;
-      if (word) wpre[g * 32 + lane] = running + pre;
-      // balanced extraction: rank r of the group belongs to lane r % 32, four ranks in flight
-      for (u32 r0 = 0; r0 < T; r0 += 128) {
-        u32 jj[4];
-        float vv[4];
-        bool act[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const u32 r = r0 + q * 32 + lane;
-          act[q] = r < T;
-          const u32 rr = act[q] ? r : T - 1;
-          u32 lo = 0;  // the last word whose exclusive prefix is <= rr holds rank rr
-#pragma unroll
-          for (int step = 16; step > 0; step >>= 1) {
-            const u32 cand = lo + step;
-            const u32 pc = __shfl_sync(kFull, pre, cand & 31);
-            if (cand < 32 && pc <= rr) lo = cand;
-          }
-          const u32 ww = __shfl_sync(kFull, word, lo);
-          const u32 pw = __shfl_sync(kFull, pre, lo);
-          const u32 bit = __fns(ww, 0, (int)(rr - pw) + 1);
-          jj[q] = (u32)((g * 32 + lo) << 5) + bit;
-          vv[q] = act[q] ? eps_row[jj[q]] : 0.0f;
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          if (act[q]) {
-            const size_t o = obase + running + r0 + q * 32 + lane;
-            eps_row[jj[q]] = 0.0f;  // a - a
-            p.out_idx[o] = (int32_t)jj[q];
-            p.out_val[o] = vv[q];
-            p.cur_idx[o] = (int32_t)jj[q];
-            p.cur_val[o] = vv[q];
-          }
-        }
-      }
-      running += T;
-    }
+  // ---- emission: ordered walk of the mask.  A block owns a contiguous run of 8-word units and
+  //      works through it in chunks of kEmitUnits; winners are dealt to threads by rank, so a
+  //      region dense with winners costs no more than the same winners spread out ----
+  __syncthreads();
+  u32* s_up = sh.hist;  // hist and spare are contiguous: exclusive winner prefix per unit of the chunk
+  const int64_t nchunks = (bu1 - bu0 + kEmitUnits - 1) / kEmitUnits;
+  u32 block_total = 0;
+  u32 chunk_total = 0;
+  for (int64_t ch = 0; ch < nchunks; ++ch) {
+    chunk_total = emit_count_chunk(sh, mask, bu0 + ch * kEmitUnits, bu1, s_up);
+    block_total += chunk_total;
   }
-  cl.sync();  // no block leaves while a peer may still read its shared memory
+  if (tid == 0) btot[rk] = block_total;
+  cl.sync();  // (3) per-block totals exchanged
+  u32 running = 0, all_total = 0;
+  for (u32 c = 0; c < CS; ++c) {
+    const u32 t = __ldcg(&btot[c]);
+    if (c < rk) running += t;
+    all_total += t;
+  }
+  if (all_total != k) {
+    if (rk == 0 && tid == 0) atomicOr(&p.gctl->err, kErrCountMismatch);
+    return;
+  }
+  u32* upre = p.uprefix + (size_t)n * (p.W >> 3);
+  for (int64_t ch = 0; ch < nchunks; ++ch) {
+    const int64_t cu0 = bu0 + ch * kEmitUnits;
+    const int64_t cu1 = cu0 + kEmitUnits < bu1 ? cu0 + kEmitUnits : bu1;
+    if (nchunks > 1) chunk_total = emit_count_chunk(sh, mask, cu0, bu1, s_up);  // else s_up is still valid
+    const int nu = (int)(cu1 - cu0);
+    for (int u = tid; u < nu; u += blockDim.x) upre[cu0 + u] = running + s_up[u];
+    // four ranks per thread in flight
+    for (u32 r0 = 0; r0 < chunk_total; r0 += 4 * blockDim.x) {
+      u32 jj[4];
+      float vv[4];
+      uint4 wx[4], wy[4];
+      u32 rel[4];
+      int64_t un[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const u32 r = r0 + q * blockDim.x + tid;
+        const u32 rr = r < chunk_total ? r : chunk_total - 1;
+        int lo = 0, hi = nu;  // last unit whose exclusive prefix is <= rr
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (s_up[mid] <= rr) lo = mid; else hi = mid;
+        }
+        un[q] = cu0 + lo;
+        rel[q] = rr - s_up[lo];
+        wx[q] = __ldcg(reinterpret_cast<const uint4*>(mask + un[q] * 8));
+        wy[q] = __ldcg(reinterpret_cast<const uint4*>(mask + un[q] * 8 + 4));
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const u32 r = r0 + q * blockDim.x + tid;
+        const u32 w[8] = {wx[q].x, wx[q].y, wx[q].z, wx[q].w, wy[q].x, wy[q].y, wy[q].z, wy[q].w};
+        u32 left = rel[q], word = 0, wi = 0;
+        bool found = false;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const u32 pc = __popc(w[i]);
+          if (!found && left < pc) { word = w[i]; wi = (u32)i; found = true; }
+          if (!found) left -= pc;
+        }
+        const u32 bit = __fns(word, 0, (int)left + 1);
+        jj[q] = (u32)((un[q] * 8 + wi) << 5) + (bit & 31u);
+        vv[q] = r < chunk_total ? eps_row[jj[q]] : 0.0f;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const u32 r = r0 + q * blockDim.x + tid;
+        if (r < chunk_total) {
+          const size_t o = obase + running + r;
+          eps_row[jj[q]] = 0.0f;  // a - a
+          p.out_idx[o] = (int32_t)jj[q];
+          p.out_val[o] = vv[q];
+          p.cur_idx[o] = (int32_t)jj[q];
+          p.cur_val[o] = vv[q];
+        }
+      }
+    }
+    running += chunk_total;
+    __syncthreads();  // s_up is rewritten by the next chunk
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
 // k_aggregate: g = sum_n omega_n * ghat_n with the workers added in the order n = 0..N-1.
 // One thread per pair sent this round: the pair of the highest-numbered worker that sent index j
-// owns g[j]; it looks the lower workers' values up (mask word, prefix count, value) and adds them
+// owns g[j]; it looks the lower workers' values up (mask unit, prefix count, value) and adds them
 // in order.  One thread per pair of the previous round clears g[j] if nobody sent j now.
 // ---------------------------------------------------------------------------------------------
 struct AggArgs {
@@ -904,7 +946,7 @@ struct AggArgs {
   const float* cur_val;
   const int32_t* prev_idx;
   const u32* bitmask;
-  const u32* wprefix;
+  const u32* uprefix;
   int64_t W;
   const float* omega;
   int has_prev;
@@ -913,6 +955,7 @@ struct AggArgs {
 __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
   const int64_t npairs = p.k * p.N;
   const int64_t total = p.has_prev ? 2 * npairs : npairs;
+  const int64_t U = p.W >> 3;
   for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
        t += (int64_t)gridDim.x * blockDim.x) {
     if (t >= npairs) {  // a pair of the previous round
@@ -933,6 +976,8 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
     const int n = (int)(t / p.k);
     const int32_t j = p.cur_idx[t];
     const size_t wi = (size_t)(j >> 5);
+    const size_t ui = wi >> 3;
+    const int wsub = (int)(wi & 7);
     const u32 bm = 1u << (j & 31);
     // a higher-numbered worker that sent j owns it
     bool owned = true;
@@ -945,21 +990,35 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
     }
     if (!owned) continue;
     float sum = 0.0f;
-    for (int m0 = 0; m0 < n; m0 += 8) {
-      u32 w[8], pre[8];
+    for (int m0 = 0; m0 < n; m0 += 4) {
+      uint4 x[4], y[4];
+      u32 pre[4];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
+      for (int u = 0; u < 4; ++u) {
         const bool in = m0 + u < n;
-        w[u] = in ? p.bitmask[(size_t)(m0 + u) * p.W + wi] : 0u;
-        pre[u] = in ? p.wprefix[(size_t)(m0 + u) * p.W + wi] : 0u;
+        const u32* unit = p.bitmask + (size_t)(m0 + u) * p.W + ui * 8;
+        x[u] = in ? *reinterpret_cast<const uint4*>(unit) : make_uint4(0, 0, 0, 0);
+        y[u] = in ? *reinterpret_cast<const uint4*>(unit + 4) : make_uint4(0, 0, 0, 0);
+        pre[u] = in ? p.uprefix[(size_t)(m0 + u) * U + ui] : 0u;
       }
-      float v[8];
+      float v[4];
+      bool has[4];
 #pragma unroll
-      for (int u = 0; u < 8; ++u)
-        v[u] = (w[u] & bm) ? p.cur_val[(size_t)(m0 + u) * p.k + pre[u] + __popc(w[u] & (bm - 1u))] : 0.0f;
+      for (int u = 0; u < 4; ++u) {
+        const u32 w[8] = {x[u].x, x[u].y, x[u].z, x[u].w, y[u].x, y[u].y, y[u].z, y[u].w};
+        u32 rank = pre[u], mine = 0;
 #pragma unroll
-      for (int u = 0; u < 8; ++u)
-        if (w[u] & bm) sum = __fadd_rn(sum, __fmul_rn(p.omega[m0 + u], v[u]));
+        for (int i = 0; i < 8; ++i) {
+          if (i < wsub) rank += __popc(w[i]);
+          if (i == wsub) mine = w[i];
+        }
+        has[u] = (mine & bm) != 0u;
+        rank += __popc(mine & (bm - 1u));
+        v[u] = has[u] ? p.cur_val[(size_t)(m0 + u) * p.k + rank] : 0.0f;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (has[u]) sum = __fadd_rn(sum, __fmul_rn(p.omega[m0 + u], v[u]));
     }
     sum = __fadd_rn(sum, __fmul_rn(p.omega[n], p.cur_val[t]));
     p.g[j] = sum;
@@ -973,7 +1032,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   int64_t ld, W, capA, stride;
-  size_t off_eps, off_g, off_mask, off_ctl, off_gctl, zero_end, off_wprefix, off_idx[2], off_val[2],
+  size_t off_eps, off_g, off_mask[2], off_ctl, off_gctl, zero_end, off_uprefix, off_ghist, off_btot, off_idx[2], off_val[2],
       off_ovr_key, off_ovr_comp, off_candA, off_candB, off_omega, off_stage_g, off_stage_idx,
       off_stage_val, total;
 };
@@ -1005,11 +1064,14 @@ Layout make_layout(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
   // state that creation and reset clear to zero comes first
   L.off_eps = take((size_t)N * L.ld * 4);
   L.off_g = take(align_up((size_t)d, 64) * 4);
-  L.off_mask = take((size_t)N * L.W * 4);
+  L.off_mask[0] = take((size_t)N * L.W * 4);
+  L.off_mask[1] = take((size_t)N * L.W * 4);
   L.off_ctl = take((size_t)N * sizeof(WorkerCtl));
   L.off_gctl = take(sizeof(GlobalCtl));
   L.zero_end = o;
-  L.off_wprefix = take((size_t)N * L.W * 4);
+  L.off_uprefix = take((size_t)N * (L.W / 8) * 4);
+  L.off_ghist = take((size_t)N * 4 * kBins * 4);
+  L.off_btot = take((size_t)N * 2 * kMaxCluster * 4);
   for (int i = 0; i < 2; ++i) {
     L.off_idx[i] = take((size_t)N * k * 4);
     L.off_val[i] = take((size_t)N * k * 4);
@@ -1101,22 +1163,26 @@ void post_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int N, int 
   cfg->numAttrs = 1;
 }
 
-// Blocks per worker for k_post: as many as keep all N clusters resident at once, a power of two,
-// at most 16 (sizes above 8 need the non-portable opt-in), and only what the device can schedule.
-int choose_cluster(int N, int num_sms) {
-  int want = 16;
-  while (want > 1 && N * want > num_sms) want >>= 1;
+// Blocks per worker for k_post: the largest power of two up to 16 (sizes above 8 need the
+// non-portable opt-in) for which the device keeps all N clusters resident at once; failing that,
+// the largest size it can schedule at all.
+int choose_cluster(int N) {
   cudaFuncSetAttribute(k_post, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   cudaGetLastError();
-  for (int cs = want; cs > 1; cs >>= 1) {
+  int schedulable = 1;
+  for (int cs = kMaxCluster; cs > 1; cs >>= 1) {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     post_config(&cfg, attr, N, cs, nullptr);
     int nclusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&nclusters, k_post, &cfg) == cudaSuccess && nclusters >= 1) return cs;
-    cudaGetLastError();
+    if (cudaOccupancyMaxActiveClusters(&nclusters, k_post, &cfg) != cudaSuccess) {
+      cudaGetLastError();
+      continue;
+    }
+    if (nclusters >= N) return cs;  // all workers' clusters run at once
+    if (nclusters >= 1 && schedulable == 1) schedulable = cs;
   }
-  return 1;
+  return schedulable;
 }
 
 }  // namespace
@@ -1181,7 +1247,7 @@ int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const reg
   c->ws = static_cast<char*>(workspace);
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->num_sms = sms > 0 ? sms : 148;
-  c->cluster = choose_cluster(N, c->num_sms);
+  c->cluster = choose_cluster(N);
   float* om = static_cast<float*>(malloc(sizeof(float) * N));
   if (!om) { free(c); return REGTOPK_ERR_INVALID_ARG; }
   for (int n = 0; n < N; ++n) om[n] = params->omega ? params->omega[n] : 1.0f / (float)N;
@@ -1215,6 +1281,7 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   sa.k = c->k;
   sa.k_target = use_marks ? (2 * c->k < c->d ? 2 * c->k : c->d) : c->k;
   sa.ctl = at<WorkerCtl>(c, L.off_ctl); sa.gctl = at<GlobalCtl>(c, L.off_gctl);
+  sa.ghist = at<u32>(c, L.off_ghist);
   sa.force_dense = (c->flags & REGTOPK_FLAG_FORCE_DENSE_SELECT) ? 1 : 0;
   if (bf16) k_sample_cutoff<true><<<c->N, kBlockSel, sample_smem(), c->stream>>>(sa);
   else k_sample_cutoff<false><<<c->N, kBlockSel, sample_smem(), c->stream>>>(sa);
@@ -1237,10 +1304,12 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   pa.omega = at<float>(c, L.off_omega); pa.mu = c->mu;
   pa.ovr_key = at<u32>(c, L.off_ovr_key); pa.ovr_comp = at<u64>(c, L.off_ovr_comp);
   pa.candA = at<u64>(c, L.off_candA); pa.candB = at<u64>(c, L.off_candB); pa.capA = L.capA; pa.stride = L.stride;
-  pa.bitmask = at<u32>(c, L.off_mask); pa.wprefix = at<u32>(c, L.off_wprefix); pa.W = L.W;
+  pa.ghist = at<u32>(c, L.off_ghist); pa.btot = at<u32>(c, L.off_btot);
+  pa.mask_old = at<u32>(c, L.off_mask[prev]); pa.mask_new = at<u32>(c, L.off_mask[c->cur]);
+  pa.uprefix = at<u32>(c, L.off_uprefix); pa.W = L.W;
   pa.out_idx = out_idx; pa.out_val = out_val;
   pa.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); pa.cur_val = at<float>(c, L.off_val[c->cur]);
-  pa.use_marks = use_marks; pa.has_prev = has_prev;
+  pa.use_marks = use_marks; pa.has_stale = c->round >= 2;
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[1];
   post_config(&cfg, attr, c->N, c->cluster, c->stream);
@@ -1261,7 +1330,7 @@ int regtopk_aggregate(regtopk_ctx* c, float* out_g) {
   a.g = at<float>(c, L.off_g); a.N = c->N; a.k = c->k;
   a.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); a.cur_val = at<float>(c, L.off_val[c->cur]);
   a.prev_idx = at<int32_t>(c, L.off_idx[c->cur ^ 1]);
-  a.bitmask = at<u32>(c, L.off_mask); a.wprefix = at<u32>(c, L.off_wprefix); a.W = L.W;
+  a.bitmask = at<u32>(c, L.off_mask[c->cur]); a.uprefix = at<u32>(c, L.off_uprefix); a.W = L.W;
   a.omega = at<float>(c, L.off_omega);
   a.has_prev = c->round >= 1;
   const int64_t threads = (a.has_prev ? 2 : 1) * c->k * (int64_t)c->N;
