@@ -15,7 +15,7 @@
 //                     zeroing the residual there.  If the cutoff guess was too high or the list
 //                     overflowed, the same cluster runs an exact radix select over the whole row.
 //   k_aggregate       server sum in worker order, one thread per sent pair, ranks looked up through
-//                     the per-unit prefix counts written during emission
+//                     the prefix counts written during emission
 //
 // The selection key of an entry is the bit pattern of its non-negative binary32 score, which orders
 // like the score; the 64-bit composite (key << 32 | ~index) orders like (score descending, index
@@ -45,13 +45,15 @@ namespace {
 typedef unsigned long long u64;
 typedef uint32_t u32;
 
-constexpr int kSampleSectors = 4096;       // 32-byte sectors sampled per worker
+constexpr int kSampleSectors = 8192;       // 32-byte sectors sampled per worker
 constexpr int kSampleMax = kSampleSectors * 8;
-constexpr int kBlockSel = 1024;            // threads of the per-worker kernels
+constexpr int kBlockSel = 1024;            // threads per block of k_sample_cutoff
+constexpr int kBlockPost = 1024;           // threads per block of k_post
 constexpr int kStreamThreads = 256;
 constexpr int kWarpList = 256;             // per-warp staging list of k_stream (entries)
 constexpr int kBins = 4096;                // histogram bins of the select
 constexpr int kMaxCluster = 16;
+constexpr int kMaxSegments = kMaxCluster * 32;  // mask segments per row: one per warp of a k_post cluster
 constexpr u32 kFull = 0xFFFFFFFFu;
 
 enum : u32 { kErrCountMismatch = 1u, kErrDenseSelect = 2u, kErrRefine = 4u };
@@ -197,8 +199,16 @@ __device__ __forceinline__ float load_grad(const void* row, int64_t j) {
 
 
 // ---------------------------------------------------------------------------------------------
-// k_sample_cutoff: one block per worker.
+// k_sample_cutoff: one cluster of kSampleCluster blocks per worker.  Each block gathers its share
+// of the sample in one wave of loads and histograms the top 14 key bits (1/64-octave bins); the
+// blocks' histograms meet in global memory at the cluster barrier, and the leader reads two order
+// statistics off the merged histogram.
 // ---------------------------------------------------------------------------------------------
+constexpr int kSampleCluster = 8;
+constexpr int kSamplePerBlock = kSampleMax / kSampleCluster;  // 8192: eight per thread
+constexpr int kSampleBins = 16384;
+constexpr int kSampleShift = 17;  // key >> 17: sign-less exponent and six mantissa bits
+
 struct SampleArgs {
   const void* grads;
   int64_t grad_ld;
@@ -208,25 +218,35 @@ struct SampleArgs {
   int64_t k;
   int64_t k_target;  // entries the cutoff should leave above it (k, or 2k when overrides can demote)
   WorkerCtl* ctl;
-  GlobalCtl* gctl;
-  u32* ghist;  // [N][4][kBins], cleared here for k_post
+  u32* ghist;  // [N][4][kBins] histograms of k_post, cleared here
+  u32* shist;  // [N][kSampleBins] histogram of this kernel; zero on entry (k_post clears it again)
   int force_dense;
 };
 
+// Add a block's histogram to the cluster's in global memory (non-empty bins only).
+__device__ __forceinline__ void flush_hist(const u32* s_hist, u32* g_hist, int nbins) {
+  for (int i = threadIdx.x; i < nbins; i += blockDim.x) {
+    const u32 v = s_hist[i];
+    if (v) atomicAdd(&g_hist[i], v);
+  }
+}
+
 template <bool BF16>
 __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
-  extern __shared__ u32 s_dyn[];
-  u32* s_keys = s_dyn;               // kSampleMax
-  u32* s_hist = s_dyn + kSampleMax;  // kBins
+  extern __shared__ u32 s_hist[];  // kSampleBins
   __shared__ u32 s_scan[33];
   __shared__ u32 s_res[3];
-  const int n = blockIdx.x;
+  cg::cluster_group cl = cg::this_cluster();
+  const u32 rk = cl.block_rank();
+  const int n = blockIdx.x / kSampleCluster;
   const int tid = threadIdx.x;
   WorkerCtl* ctl = p.ctl + n;
+  u32* shist = p.shist + (size_t)n * kSampleBins;
 
-  for (int i = tid; i < 4 * kBins; i += blockDim.x) p.ghist[(size_t)n * 4 * kBins + i] = 0;
-  if (p.force_dense) {
-    if (tid == 0) {
+  for (int i = rk * blockDim.x + tid; i < 4 * kBins; i += kSampleCluster * blockDim.x)
+    p.ghist[(size_t)n * 4 * kBins + i] = 0;
+  if (p.force_dense) {  // the same in every block: nobody reaches a barrier
+    if (rk == 0 && tid == 0) {
       ctl->cutoff = kFull;  // no key reaches it: the stream pass collects nothing
       ctl->bin_shift = 0;
       ctl->cand_count = 0;
@@ -240,38 +260,35 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
 
   const int64_t Q = (p.d + 7) >> 3;  // 8-element sectors in the row
   const bool all = Q <= kSampleSectors;
-  const int nsect = all ? (int)Q : kSampleSectors;
+  const int nslots = (all ? (int)Q : kSampleSectors) * 8;
   const int M = all ? (int)p.d : kSampleMax;  // samples that lie inside the row
   const float* eps_row = p.eps + (size_t)n * p.ld;
   const char* grow = static_cast<const char*>(p.grads) + (size_t)n * p.grad_ld * (BF16 ? 2 : 4);
 
-  for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
-  __syncthreads();
-  // eight independent sample loads in flight per thread
-  for (int i0 = 0; i0 < nsect * 8; i0 += 8 * kBlockSel) {
+  {  // this block's slots: [rk * kSamplePerBlock, +kSamplePerBlock), eight per thread, one wave of loads
     float e[8], g[8];
     bool ok[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const int i = i0 + u * kBlockSel + tid;
-      const int s = i >> 3;
-      const int64_t q = all ? s : (int64_t)(((u64)s * (u64)Q) / (u64)kSampleSectors);
+      const int i = (int)rk * kSamplePerBlock + u * kBlockSel + tid;
+      const int sct = i >> 3;
+      const int64_t q = all ? sct : (int64_t)(((u64)sct * (u64)Q) / (u64)kSampleSectors);
       const int64_t j = q * 8 + (i & 7);
-      ok[u] = i < nsect * 8 && j < p.d;
+      ok[u] = i < nslots && j < p.d;
       e[u] = ok[u] ? eps_row[j] : 0.0f;
       g[u] = ok[u] ? load_grad<BF16>(grow, j) : 0.0f;
     }
+    for (int i = tid; i < kSampleBins; i += blockDim.x) s_hist[i] = 0;  // while the loads are in flight
+    __syncthreads();
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int i = i0 + u * kBlockSel + tid;
-      u32 key = kFull;  // marks a slot outside the row
-      if (ok[u]) {
-        key = __float_as_uint(__fadd_rn(e[u], g[u])) & 0x7FFFFFFFu;
-        atomicAdd(&s_hist[key >> 19], 1u);
-      }
-      if (i < nsect * 8) s_keys[i] = key;
-    }
+    for (int u = 0; u < 8; ++u)
+      if (ok[u]) atomicAdd(&s_hist[(__float_as_uint(__fadd_rn(e[u], g[u])) & 0x7FFFFFFFu) >> kSampleShift], 1u);
   }
+  __syncthreads();
+  flush_hist(s_hist, shist, kSampleBins);
+  cl.sync();  // histogram of the whole sample complete
+  if (rk != 0) return;
+  for (int i = tid; i < kSampleBins; i += blockDim.x) s_hist[i] = __ldcg(&shist[i]);
   __syncthreads();
 
   // Ranks to read off the sample.  The number of sample points above a quantile is close to Poisson
@@ -286,28 +303,15 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
 
   // upper end of the key range the select should resolve finely: the k-th largest score cannot
   // exceed the k-th largest |a|, estimated from above by the sample's r_hi-th largest
-  block_find_from_top(s_hist, kBins, r_hi, s_scan, s_res);
-  u32 hi_key = s_res[0] == kFull ? 0x7F7FFFFFu : (((s_res[0] + 1u) << 19) - 1u);
+  block_find_from_top(s_hist, kSampleBins, r_hi, s_scan, s_res);
+  u32 hi_key = s_res[0] == kFull ? 0x7F7FFFFFu : (((s_res[0] + 1u) << kSampleShift) - 1u);
   __syncthreads();
   if (r_hi_d < 1.0) hi_key = hi_key < 0x7F000000u ? hi_key + (1u << 23) : 0x7F7FFFFFu;  // an octave of slack
 
-  u32 cutoff = 0;
+  u32 cutoff = 0;  // lower edge of the bin that holds the r_lo-th largest sample
   if (r_lo <= (u32)M) {
-    block_find_from_top(s_hist, kBins, r_lo, s_scan, s_res);
-    const u32 b1 = s_res[0], above1 = s_res[1];
-    __syncthreads();
-    if (b1 != kFull) {
-      for (int i = tid; i < 1024; i += blockDim.x) s_hist[i] = 0;
-      __syncthreads();
-      for (int i = tid; i < nsect * 8; i += blockDim.x) {
-        const u32 key = s_keys[i];
-        if (key != kFull && (key >> 19) == b1) atomicAdd(&s_hist[(key >> 9) & 1023u], 1u);
-      }
-      __syncthreads();
-      block_find_from_top(s_hist, 1024, r_lo - above1, s_scan, s_res);
-      const u32 b2 = s_res[0];
-      cutoff = (b1 << 19) | ((b2 == kFull ? 0u : b2) << 9);
-    }
+    block_find_from_top(s_hist, kSampleBins, r_lo, s_scan, s_res);
+    if (s_res[0] != kFull) cutoff = s_res[0] << kSampleShift;
   }
   if (tid == 0) {
     const u32 range = hi_key > cutoff ? hi_key - cutoff : 0u;
@@ -477,10 +481,13 @@ struct PostArgs {
   int64_t capA;
   int64_t stride;  // capA + k: what one histogram bin can hold (all candidates plus all overrides)
   u32* ghist;      // [N][4][kBins] cluster-wide histograms, zeroed by k_sample_cutoff
+  u32* shist;      // [N][kSampleBins] histogram of k_sample_cutoff, cleared here for the next round
   u32* btot;       // [N][2][kMaxCluster] per-block totals
   const u32* mask_old;  // [N][W] last round's mask (marks the previous support)
   u32* mask_new;   // [N][W] this round's mask; on entry it holds the mask of two rounds ago
-  u32* uprefix;    // [N][W/8] winners before each 8-word unit of the mask (rank directory for k_aggregate)
+  u32* qprefix;    // [N][W/4] mask bits before each quad (4 words) within its segment
+  u32* segtot;     // [N][kMaxSegments] mask bits of each segment
+  u32* segbase;    // [N][kMaxSegments] mask bits before each segment (written for k_aggregate)
   int64_t W;       // words per row, a multiple of 32
   int32_t* out_idx;
   float* out_val;
@@ -508,14 +515,6 @@ __device__ __forceinline__ void set_winner(u32* mask, u32 idx) {
 __device__ __forceinline__ u32 select_bin(u32 key, u32 cutoff, u32 shift) {
   const u32 b = (key - cutoff) >> shift;
   return b < (u32)(kBins - 1) ? b : (u32)(kBins - 1);
-}
-
-// Add this block's histogram to the cluster's in global memory (non-empty bins only).
-__device__ __forceinline__ void flush_hist(const u32* s_hist, u32* g_hist) {
-  for (int i = threadIdx.x; i < kBins; i += blockDim.x) {
-    const u32 v = s_hist[i];
-    if (v) atomicAdd(&g_hist[i], v);
-  }
 }
 
 // After the cluster barrier: every block loads the cluster's histogram and finds the bin of the
@@ -548,7 +547,7 @@ __device__ __forceinline__ u32 dense_key(const PostArgs& p, int n, int64_t j) {
   return __float_as_uint(p.eps[(size_t)n * p.ld + j]) & 0x7FFFFFFFu;
 }
 
-// One block: among list[0..count) (count <= 1024, unique composites) set the `need` largest as
+// One block: among list[0..count) (count <= blockDim.x, unique composites) set the `need` largest as
 // winners, but only those whose mask word lies in [w0, w1) (the caller's share of the mask).
 __device__ void refine_small(PostShared& sh, u32* mask, const u64* list, u32 count, u32 need,
                              int64_t w0, int64_t w1) {
@@ -572,94 +571,43 @@ __device__ void refine_small(PostShared& sh, u32* mask, const u64* list, u32 cou
   __syncthreads();
 }
 
-// Leader block only: the `need` largest composites of list[0..count), any count, by radix passes
-// over all 64 bits.  `other` (same capacity) is the second buffer.
-__device__ void refine_large(PostShared& sh, u32* mask, GlobalCtl* gctl, u64* list, u64* other,
-                             u32 count, u32 need) {
+// Leader block only: the `need` largest composites of list[0..count), any count (long runs of equal
+// keys end up here).  Eight histogram passes over the list fix the need-th largest composite byte by
+// byte, without moving the list; a last pass sets everything at or above it.
+__device__ void refine_large(PostShared& sh, u32* mask, GlobalCtl* gctl, const u64* list, u32 count,
+                             u32 need) {
   const int tid = threadIdx.x;
-  u64* src = list;
-  u64* dst = other;
-  u32 nsrc = count;
+  if (need == 0) return;
+  u64 prefix = 0ull;  // the bytes of the need-th largest composite fixed so far
   for (int shift = 56; shift >= 0; shift -= 8) {
-    if (need == 0) return;
-    if (need >= nsrc) break;
     for (int i = tid; i < 256; i += blockDim.x) sh.hist[i] = 0;
-    if (tid == 0) sh.cnt = 0;
     __syncthreads();
-    for (u32 i = tid; i < nsrc; i += blockDim.x) atomicAdd(&sh.hist[(u32)(__ldcg(&src[i]) >> shift) & 255u], 1u);
+    for (u32 i = tid; i < count; i += blockDim.x) {
+      const u64 c = __ldcg(&list[i]);
+      if (shift == 56 || (c >> (shift + 8)) == prefix) atomicAdd(&sh.hist[(u32)(c >> shift) & 255u], 1u);
+    }
     __syncthreads();
     block_find_from_top(sh.hist, 256, need, sh.scan, sh.fres);
     const u32 b = sh.fres[0], above = sh.fres[1];
     __syncthreads();
-    if (b == kFull) {  // cannot happen: need <= nsrc
+    if (b == kFull) {  // cannot happen while need <= count
       if (tid == 0) atomicOr(&gctl->err, kErrRefine);
       return;
     }
-    const u32 iters = (nsrc + blockDim.x - 1) / blockDim.x;
-    for (u32 it = 0; it < iters; ++it) {
-      const u32 i = it * blockDim.x + tid;
-      u64 c = 0ull;
-      u32 dg = 0;
-      if (i < nsrc) {
-        c = __ldcg(&src[i]);
-        dg = (u32)(c >> shift) & 255u;
-        if (dg > b) set_winner(mask, composite_idx(c));
-      }
-      const bool inbin = i < nsrc && dg == b;
-      const u32 pos = warp_reserve(inbin, &sh.cnt);
-      if (inbin) dst[pos] = c;
-    }
-    __syncthreads();
     need -= above;
-    nsrc = sh.cnt;
-    __syncthreads();
-    u64* t = src; src = dst; dst = t;
+    prefix = (prefix << 8) | (u64)b;
   }
-  if (need >= nsrc) {
-    for (u32 i = tid; i < nsrc; i += blockDim.x) set_winner(mask, composite_idx(__ldcg(&src[i])));
-  } else if (need != 0) {
-    if (tid == 0) atomicOr(&gctl->err, kErrRefine);  // all bits consumed: composites were not unique
+  for (u32 i = tid; i < count; i += blockDim.x) {
+    const u64 c = __ldcg(&list[i]);
+    if (c >= prefix) set_winner(mask, composite_idx(c));
   }
 }
 
-constexpr int kEmitUnits = 2 * kBins;  // 8-word units per emission chunk (the shared prefix array holds one word each)
-
-// Count the winners of the units [cu0, min(cu0 + kEmitUnits, bu1)) of a mask row: s_up[u] receives
-// the winners before unit u within the chunk; returns the chunk's total.  A thread owns 8 consecutive
-// units.  Every thread of the block must call it.
-__device__ u32 emit_count_chunk(PostShared& sh, const u32* mask, int64_t cu0, int64_t bu1, u32* s_up) {
-  const int tid = threadIdx.x;
-  u32 c[8];
-  u32 sum = 0;
-  uint4 x[8], y[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int64_t u = cu0 + tid * 8 + i;
-    x[i] = make_uint4(0, 0, 0, 0);
-    y[i] = x[i];
-    if (u < bu1) {
-      x[i] = __ldcg(reinterpret_cast<const uint4*>(mask + u * 8));
-      y[i] = __ldcg(reinterpret_cast<const uint4*>(mask + u * 8 + 4));
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    c[i] = __popc(x[i].x) + __popc(x[i].y) + __popc(x[i].z) + __popc(x[i].w) + __popc(y[i].x) +
-           __popc(y[i].y) + __popc(y[i].z) + __popc(y[i].w);
-    sum += c[i];
-  }
-  u32 total;
-  u32 run = block_excl_scan(sum, sh.scan, &total);
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    s_up[tid * 8 + i] = run;
-    run += c[i];
-  }
-  __syncthreads();
-  return total;
+__device__ __forceinline__ u32 popc4(const uint4& v) {
+  return (u32)(__popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w));
 }
 
-__global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
+__global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
   __shared__ __align__(16) PostShared sh;
   cg::cluster_group cl = cg::this_cluster();
   const u32 CS = cl.num_blocks(), rk = cl.block_rank();
@@ -687,11 +635,18 @@ __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
   const bool overflow = (u64)cand_count > (u64)p.capA;
   const u32 ncand = overflow ? (u32)p.capA : cand_count;
   const u32 novr = p.use_marks ? k : 0u;
-  // this block's share of the mask for the emission: units of 8 words
+  // The mask row is cut into one segment of 8-word units per warp of the cluster; a block's share
+  // is the segments of its warps.  The refinement and the emission both use this partition, so a
+  // block only ever reads mask words whose last writers it has met at a barrier.
   const int64_t U = p.W >> 3;
-  const int64_t bu0 = (int64_t)(((u64)rk * (u64)U) / CS), bu1 = (int64_t)(((u64)(rk + 1) * (u64)U) / CS);
+  const int nw = blockDim.x >> 5;
+  const u32 nseg = CS * (u32)nw;
+  const int64_t seg_units = (U + nseg - 1) / nseg;
+  const int64_t su0 = (int64_t)rk * nw * seg_units < U ? (int64_t)rk * nw * seg_units : U;
+  const int64_t su1 = (int64_t)(rk + 1) * nw * seg_units < U ? (int64_t)(rk + 1) * nw * seg_units : U;
 
   for (int i = tid; i < kBins; i += blockDim.x) sh.hist[i] = 0;
+  for (u32 i = first_t; i < (u32)kSampleBins; i += stride_t) p.shist[(size_t)n * kSampleBins + i] = 0;
   __syncthreads();
   // ---- one fused sweep, so that the independent loads of its three jobs are in flight together:
   //   (a) the mask buffer of this round still holds the mask of two rounds ago: clear those words;
@@ -701,47 +656,63 @@ __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
   {
     const float w = p.omega[n];
     const u32 span = !dense && ncand > k ? ncand : k;
-    for (u32 i = first_t; i < span; i += stride_t) {
-      const bool in_k = i < k;
-      const bool do_ovr = in_k && p.use_marks;
-      const bool do_cand = !dense && i < ncand;
-      // first wave of loads
-      const int32_t stale = (in_k && p.has_stale) ? p.cur_idx[obase + i] : 0;
-      const int32_t j = do_ovr ? prev_idx[i] : 0;
-      const float ap = do_ovr ? prev_val[i] : 0.0f;
-      const u64 c = do_cand ? A[i] : 0ull;
-      // second wave, dependent on the first
-      const float a = do_ovr ? eps_row[j] : 0.0f;
-      const float G = do_ovr ? p.g_prev[j] : 0.0f;
-      const u32 cidx = composite_idx(c);
-      const u32 mword = (do_cand && p.use_marks) ? mask_old[cidx >> 5] : 0u;
-      if (in_k && p.has_stale) mask[(u32)stale >> 5] = 0u;
-      if (do_ovr) {
-        const float num = __fsub_rn(G, __fmul_rn(w, ap));
-        const float den = __fmul_rn(w, a);
-        float m = 1.0f;
-        if (den != 0.0f) {
-          const float delta = __fdiv_rn(num, den);
-          const float r = fabsf(__fadd_rn(1.0f, delta));
-          m = tanh_fixed(__fdiv_rn(r, p.mu));
-        }
-        const u32 key = __float_as_uint(__fmul_rn(fabsf(a), m));
-        const u64 oc = key >= cutoff ? make_composite(key, (u32)j) : 0ull;
-        okey[i] = key;
-        O[i] = oc;
-        if (!dense && oc) atomicAdd(&sh.hist[select_bin(key, cutoff, bshift)], 1u);
+    constexpr int kP0 = 4;  // items per thread in flight
+    for (u32 i0 = first_t; i0 < span; i0 += kP0 * stride_t) {
+      bool in_k[kP0], do_ovr[kP0], do_cand[kP0];
+      int32_t stale[kP0], j[kP0];
+      float ap[kP0], a[kP0], G[kP0];
+      u64 c[kP0];
+      u32 mword[kP0];
+#pragma unroll
+      for (int q = 0; q < kP0; ++q) {  // first wave of loads
+        const u32 i = i0 + q * stride_t;
+        in_k[q] = i < k;
+        do_ovr[q] = in_k[q] && p.use_marks;
+        do_cand[q] = !dense && i < ncand;
+        stale[q] = (in_k[q] && p.has_stale) ? p.cur_idx[obase + i] : 0;
+        j[q] = do_ovr[q] ? prev_idx[i] : 0;
+        ap[q] = do_ovr[q] ? prev_val[i] : 0.0f;
+        c[q] = do_cand[q] ? A[i] : 0ull;
       }
-      if (do_cand) {
-        if ((mword >> (cidx & 31)) & 1u) A[i] = 0ull;
-        else atomicAdd(&sh.hist[select_bin((u32)(c >> 32), cutoff, bshift)], 1u);
+#pragma unroll
+      for (int q = 0; q < kP0; ++q) {  // second wave, dependent on the first
+        a[q] = do_ovr[q] ? eps_row[j[q]] : 0.0f;
+        G[q] = do_ovr[q] ? p.g_prev[j[q]] : 0.0f;
+        mword[q] = (do_cand[q] && p.use_marks) ? mask_old[composite_idx(c[q]) >> 5] : 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < kP0; ++q) {
+        const u32 i = i0 + q * stride_t;
+        if (in_k[q] && p.has_stale) mask[(u32)stale[q] >> 5] = 0u;
+        if (do_ovr[q]) {
+          const float num = __fsub_rn(G[q], __fmul_rn(w, ap[q]));
+          const float den = __fmul_rn(w, a[q]);
+          float m = 1.0f;
+          if (den != 0.0f) {
+            const float delta = __fdiv_rn(num, den);
+            const float r = fabsf(__fadd_rn(1.0f, delta));
+            m = tanh_fixed(__fdiv_rn(r, p.mu));
+          }
+          const u32 key = __float_as_uint(__fmul_rn(fabsf(a[q]), m));
+          const u64 oc = key >= cutoff ? make_composite(key, (u32)j[q]) : 0ull;
+          okey[i] = key;
+          O[i] = oc;
+          if (!dense && oc) atomicAdd(&sh.hist[select_bin(key, cutoff, bshift)], 1u);
+        }
+        if (do_cand[q]) {
+          const u32 cidx = composite_idx(c[q]);
+          if ((mword[q] >> (cidx & 31)) & 1u) A[i] = 0ull;
+          else atomicAdd(&sh.hist[select_bin((u32)(c[q] >> 32), cutoff, bshift)], 1u);
+        }
       }
     }
   }
   __syncthreads();
-  if (!dense) flush_hist(sh.hist, ghist);
+  if (!dense) flush_hist(sh.hist, ghist, kBins);
   cl.sync();  // (1) cluster histogram complete; stale mask words cleared; override keys written
 
   u32 b1 = kFull, above1 = 0, nvalid = 0;
+  bool took_dense = false;
   if (!dense) {
     load_and_find(sh, ghist, k, &b1, &above1, &nvalid);
     if (b1 == kFull || overflow) dense = true;  // cutoff guessed too high, or the list overflowed
@@ -768,15 +739,16 @@ __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
     cl.sync();  // (2) refinement list complete
     const u32 nB = __ldcg(&ctl->bcount);
     const u32 need = k - above1;
-    if (nB <= 1024u) {
+    if (nB <= blockDim.x) {
       // every block ranks the short list itself and sets the winners of its own share of the mask
-      refine_small(sh, mask, B, nB, need, bu0 * 8, bu1 * 8);
+      refine_small(sh, mask, B, nB, need, su0 * 8, su1 * 8);
     } else {
-      if (rk == 0) refine_large(sh, mask, p.gctl, B, A, nB, need);
+      if (rk == 0) refine_large(sh, mask, p.gctl, B, nB, need);
       cl.sync();  // (2b) the leader's winners are set
     }
   } else {
     // ---- exact selection over the whole row: three radix digits of the 31-bit key ----
+    took_dense = true;
     if (rk == 0 && tid == 0) atomicAdd(&p.gctl->dense_workers, 1ull);
     const int64_t c0 = (int64_t)(((u64)rk * (u64)p.d) / CS);
     const int64_t c1 = (int64_t)(((u64)(rk + 1) * (u64)p.d) / CS);
@@ -795,7 +767,7 @@ __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
         if (lv == 0 || (key >> (shf + widths[lv])) == prefix) atomicAdd(&sh.hist[(key >> shf) & nbm], 1u);
       }
       __syncthreads();
-      flush_hist(sh.hist, ghist + (1 + lv) * kBins);
+      flush_hist(sh.hist, ghist + (1 + lv) * kBins, kBins);
       cl.sync();
       u32 b, above, total;
       load_and_find(sh, ghist + (1 + lv) * kBins, need, &b, &above, &total);
@@ -846,96 +818,124 @@ __global__ void __launch_bounds__(kBlockSel, 1) k_post(PostArgs p) {
     cl.sync();  // every winner bit is set
   }
 
-  // ---- emission: ordered walk of the mask.  A block owns a contiguous run of 8-word units and
-  //      works through it in chunks of kEmitUnits; winners are dealt to threads by rank, so a
-  //      region dense with winners costs no more than the same winners spread out ----
+  // ---- emission.  The rank of a winner (its place in the ascending output) is the number of mask
+  //      bits before it.  (E1) every warp of the cluster owns a fixed segment of the mask row and
+  //      writes, per quad (four words, 128 coordinates), the bits before it inside the segment;
+  //      (E2) the segment totals are exchanged and scanned; (E3) every candidate whose mask bit is
+  //      set looks its rank up (segment base + quad prefix + bits before it in the quad) and writes
+  //      its pair there.  Work in E3 follows the candidate lists, which are spread evenly over the
+  //      threads, so a region dense with winners costs no more than a sparse one. ----
   __syncthreads();
-  u32* s_up = sh.hist;  // hist and spare are contiguous: exclusive winner prefix per unit of the chunk
-  const int64_t nchunks = (bu1 - bu0 + kEmitUnits - 1) / kEmitUnits;
-  u32 block_total = 0;
-  u32 chunk_total = 0;
-  for (int64_t ch = 0; ch < nchunks; ++ch) {
-    chunk_total = emit_count_chunk(sh, mask, bu0 + ch * kEmitUnits, bu1, s_up);
-    block_total += chunk_total;
+  const int lane = tid & 31, warp = tid >> 5;
+  const u32 gw = rk * (u32)nw + (u32)warp;  // this warp's segment
+  const uint4* quads = reinterpret_cast<const uint4*>(mask);
+  u32* qpre = p.qprefix + (size_t)n * (p.W >> 2);
+  {
+    const int64_t wu0 = (int64_t)gw * seg_units < U ? (int64_t)gw * seg_units : U;
+    const int64_t wu1 = wu0 + seg_units < U ? wu0 + seg_units : U;
+    uint4 nx[2], ny[2];
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+      const int64_t u = wu0 + it * 32 + lane;
+      nx[it] = u < wu1 ? __ldcg(quads + 2 * u) : make_uint4(0, 0, 0, 0);
+      ny[it] = u < wu1 ? __ldcg(quads + 2 * u + 1) : make_uint4(0, 0, 0, 0);
+    }
+    u32 running = 0;
+    for (int64_t ub = wu0; ub < wu1; ub += 64) {
+      uint4 x[2], y[2];
+#pragma unroll
+      for (int it = 0; it < 2; ++it) {
+        x[it] = nx[it];
+        y[it] = ny[it];
+        const int64_t u = ub + 64 + it * 32 + lane;  // next step's units, in flight during this step
+        nx[it] = u < wu1 ? __ldcg(quads + 2 * u) : make_uint4(0, 0, 0, 0);
+        ny[it] = u < wu1 ? __ldcg(quads + 2 * u + 1) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int it = 0; it < 2; ++it) {
+        const u32 cx = popc4(x[it]), c = cx + popc4(y[it]);
+        u32 inc = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const u32 t = __shfl_up_sync(kFull, inc, o);
+          if (lane >= o) inc += t;
+        }
+        const int64_t u = ub + it * 32 + lane;
+        const u32 pre = running + inc - c;
+        if (u < wu1) *reinterpret_cast<uint2*>(qpre + 2 * u) = make_uint2(pre, pre + cx);
+        running += __shfl_sync(kFull, inc, 31);
+      }
+    }
+    if (lane == 0) p.segtot[(size_t)n * kMaxSegments + gw] = running;
   }
-  if (tid == 0) btot[rk] = block_total;
-  cl.sync();  // (3) per-block totals exchanged
-  u32 running = 0, all_total = 0;
-  for (u32 c = 0; c < CS; ++c) {
-    const u32 t = __ldcg(&btot[c]);
-    if (c < rk) running += t;
-    all_total += t;
+  cl.sync();  // (3) segment totals and quad prefixes of the whole row are written
+  u32* s_segbase = sh.spare;  // kMaxSegments <= kBins entries
+  {
+    u32 total;
+    const u32 t = (u32)tid < nseg ? __ldcg(&p.segtot[(size_t)n * kMaxSegments + tid]) : 0u;
+    const u32 base = block_excl_scan(t, sh.scan, &total);
+    if ((u32)tid < nseg) {
+      s_segbase[tid] = base;
+      if (rk == 0) p.segbase[(size_t)n * kMaxSegments + tid] = base;  // for k_aggregate
+    }
+    __syncthreads();
+    if (total != k) {  // the same in every block
+      if (rk == 0 && tid == 0) atomicOr(&p.gctl->err, kErrCountMismatch);
+      return;
+    }
   }
-  if (all_total != k) {
-    if (rk == 0 && tid == 0) atomicOr(&p.gctl->err, kErrCountMismatch);
-    return;
-  }
-  u32* upre = p.uprefix + (size_t)n * (p.W >> 3);
-  for (int64_t ch = 0; ch < nchunks; ++ch) {
-    const int64_t cu0 = bu0 + ch * kEmitUnits;
-    const int64_t cu1 = cu0 + kEmitUnits < bu1 ? cu0 + kEmitUnits : bu1;
-    if (nchunks > 1) chunk_total = emit_count_chunk(sh, mask, cu0, bu1, s_up);  // else s_up is still valid
-    const int nu = (int)(cu1 - cu0);
-    for (int u = tid; u < nu; u += blockDim.x) upre[cu0 + u] = running + s_up[u];
-    // four ranks per thread in flight
-    for (u32 r0 = 0; r0 < chunk_total; r0 += 4 * blockDim.x) {
-      u32 jj[4];
+  for (int part = 0; part < 2; ++part) {
+    // normal path: candidates, then overrides; dense path: its k winners, nothing else
+    const u64* items = part == 0 ? A : O;
+    const u32 count = part == 0 ? (took_dense ? k : ncand) : (took_dense ? 0u : novr);
+    for (u32 i0 = first_t; i0 < count; i0 += 4 * stride_t) {
+      u64 c[4];
+      uint4 qw[4];
+      u32 qp[4];
       float vv[4];
-      uint4 wx[4], wy[4];
-      u32 rel[4];
-      int64_t un[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const u32 r = r0 + q * blockDim.x + tid;
-        const u32 rr = r < chunk_total ? r : chunk_total - 1;
-        int lo = 0, hi = nu;  // last unit whose exclusive prefix is <= rr
-        while (hi - lo > 1) {
-          const int mid = (lo + hi) >> 1;
-          if (s_up[mid] <= rr) lo = mid; else hi = mid;
-        }
-        un[q] = cu0 + lo;
-        rel[q] = rr - s_up[lo];
-        wx[q] = __ldcg(reinterpret_cast<const uint4*>(mask + un[q] * 8));
-        wy[q] = __ldcg(reinterpret_cast<const uint4*>(mask + un[q] * 8 + 4));
+        const u32 i = i0 + q * stride_t;
+        c[q] = i < count ? __ldcg(items + i) : 0ull;
       }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const u32 r = r0 + q * blockDim.x + tid;
-        const u32 w[8] = {wx[q].x, wx[q].y, wx[q].z, wx[q].w, wy[q].x, wy[q].y, wy[q].z, wy[q].w};
-        u32 left = rel[q], word = 0, wi = 0;
-        bool found = false;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const u32 pc = __popc(w[i]);
-          if (!found && left < pc) { word = w[i]; wi = (u32)i; found = true; }
-          if (!found) left -= pc;
-        }
-        const u32 bit = __fns(word, 0, (int)left + 1);
-        jj[q] = (u32)((un[q] * 8 + wi) << 5) + (bit & 31u);
-        vv[q] = r < chunk_total ? eps_row[jj[q]] : 0.0f;
+        const u32 idx = composite_idx(c[q]);
+        const bool valid = c[q] != 0ull;
+        qw[q] = valid ? __ldcg(quads + (idx >> 7)) : make_uint4(0, 0, 0, 0);
+        qp[q] = valid ? __ldcg(qpre + (idx >> 7)) : 0u;
+        vv[q] = valid ? eps_row[idx] : 0.0f;  // fetched before the bit test: most candidates near the top win
       }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const u32 r = r0 + q * blockDim.x + tid;
-        if (r < chunk_total) {
-          const size_t o = obase + running + r;
-          eps_row[jj[q]] = 0.0f;  // a - a
-          p.out_idx[o] = (int32_t)jj[q];
-          p.out_val[o] = vv[q];
-          p.cur_idx[o] = (int32_t)jj[q];
-          p.cur_val[o] = vv[q];
+        if (c[q] == 0ull) continue;
+        const u32 idx = composite_idx(c[q]);
+        const u32 w[4] = {qw[q].x, qw[q].y, qw[q].z, qw[q].w};
+        const u32 wsel = (idx >> 5) & 3u;
+        u32 before = 0, word = 0;
+#pragma unroll
+        for (int wi = 0; wi < 4; ++wi) {
+          if ((u32)wi < wsel) before += __popc(w[wi]);
+          if ((u32)wi == wsel) word = w[wi];
+        }
+        const u32 bm = 1u << (idx & 31);
+        if (word & bm) {
+          const u32 r = s_segbase[(idx >> 8) / (u32)seg_units] + qp[q] + before + __popc(word & (bm - 1u));
+          eps_row[idx] = 0.0f;  // a - a
+          p.out_idx[obase + r] = (int32_t)idx;
+          p.out_val[obase + r] = vv[q];
+          p.cur_idx[obase + r] = (int32_t)idx;
+          p.cur_val[obase + r] = vv[q];
         }
       }
     }
-    running += chunk_total;
-    __syncthreads();  // s_up is rewritten by the next chunk
   }
 }
 
 // ---------------------------------------------------------------------------------------------
 // k_aggregate: g = sum_n omega_n * ghat_n with the workers added in the order n = 0..N-1.
 // One thread per pair sent this round: the pair of the highest-numbered worker that sent index j
-// owns g[j]; it looks the lower workers' values up (mask unit, prefix count, value) and adds them
+// owns g[j]; it looks the lower workers' values up (mask quad, prefix counts, value) and adds them
 // in order.  One thread per pair of the previous round clears g[j] if nobody sent j now.
 // ---------------------------------------------------------------------------------------------
 struct AggArgs {
@@ -946,7 +946,9 @@ struct AggArgs {
   const float* cur_val;
   const int32_t* prev_idx;
   const u32* bitmask;
-  const u32* uprefix;
+  const u32* qprefix;
+  const u32* segbase;
+  int64_t seg_units;
   int64_t W;
   const float* omega;
   int has_prev;
@@ -955,7 +957,7 @@ struct AggArgs {
 __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
   const int64_t npairs = p.k * p.N;
   const int64_t total = p.has_prev ? 2 * npairs : npairs;
-  const int64_t U = p.W >> 3;
+  const int64_t Q = p.W >> 2;
   for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
        t += (int64_t)gridDim.x * blockDim.x) {
     if (t >= npairs) {  // a pair of the previous round
@@ -976,9 +978,10 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
     const int n = (int)(t / p.k);
     const int32_t j = p.cur_idx[t];
     const size_t wi = (size_t)(j >> 5);
-    const size_t ui = wi >> 3;
-    const int wsub = (int)(wi & 7);
+    const size_t qi = wi >> 2;
+    const int wsub = (int)(wi & 3);
     const u32 bm = 1u << (j & 31);
+    const size_t seg = (size_t)((int64_t)(wi >> 3) / p.seg_units);
     // a higher-numbered worker that sent j owns it
     bool owned = true;
     for (int m0 = n + 1; m0 < p.N && owned; m0 += 8) {
@@ -991,24 +994,23 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
     if (!owned) continue;
     float sum = 0.0f;
     for (int m0 = 0; m0 < n; m0 += 4) {
-      uint4 x[4], y[4];
+      uint4 x[4];
       u32 pre[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const bool in = m0 + u < n;
-        const u32* unit = p.bitmask + (size_t)(m0 + u) * p.W + ui * 8;
-        x[u] = in ? *reinterpret_cast<const uint4*>(unit) : make_uint4(0, 0, 0, 0);
-        y[u] = in ? *reinterpret_cast<const uint4*>(unit + 4) : make_uint4(0, 0, 0, 0);
-        pre[u] = in ? p.uprefix[(size_t)(m0 + u) * U + ui] : 0u;
+        x[u] = in ? *reinterpret_cast<const uint4*>(p.bitmask + (size_t)(m0 + u) * p.W + qi * 4)
+                  : make_uint4(0, 0, 0, 0);
+        pre[u] = in ? p.qprefix[(size_t)(m0 + u) * Q + qi] + p.segbase[(size_t)(m0 + u) * kMaxSegments + seg] : 0u;
       }
       float v[4];
       bool has[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const u32 w[8] = {x[u].x, x[u].y, x[u].z, x[u].w, y[u].x, y[u].y, y[u].z, y[u].w};
+        const u32 w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
         u32 rank = pre[u], mine = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < 4; ++i) {
           if (i < wsub) rank += __popc(w[i]);
           if (i == wsub) mine = w[i];
         }
@@ -1032,7 +1034,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   int64_t ld, W, capA, stride;
-  size_t off_eps, off_g, off_mask[2], off_ctl, off_gctl, zero_end, off_uprefix, off_ghist, off_btot, off_idx[2], off_val[2],
+  size_t off_eps, off_g, off_mask[2], off_ctl, off_gctl, off_shist, zero_end, off_qprefix, off_segtot, off_segbase, off_ghist, off_btot, off_idx[2], off_val[2],
       off_ovr_key, off_ovr_comp, off_candA, off_candB, off_omega, off_stage_g, off_stage_idx,
       off_stage_val, total;
 };
@@ -1068,8 +1070,11 @@ Layout make_layout(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
   L.off_mask[1] = take((size_t)N * L.W * 4);
   L.off_ctl = take((size_t)N * sizeof(WorkerCtl));
   L.off_gctl = take(sizeof(GlobalCtl));
+  L.off_shist = take((size_t)N * kSampleBins * 4);
   L.zero_end = o;
-  L.off_uprefix = take((size_t)N * (L.W / 8) * 4);
+  L.off_qprefix = take((size_t)N * (L.W / 4) * 4);
+  L.off_segtot = take((size_t)N * kMaxSegments * 4);
+  L.off_segbase = take((size_t)N * kMaxSegments * 4);
   L.off_ghist = take((size_t)N * 4 * kBins * 4);
   L.off_btot = take((size_t)N * 2 * kMaxCluster * 4);
   for (int i = 0; i < 2; ++i) {
@@ -1133,7 +1138,7 @@ int after_launch(regtopk_ctx* c) {
   return note_cuda(c, cudaGetLastError());
 }
 
-size_t sample_smem() { return (size_t)(kSampleMax + kBins) * sizeof(u32); }
+size_t sample_smem() { return (size_t)kSampleBins * sizeof(u32); }
 
 template <bool BF16, bool VEC>
 void launch_stream(regtopk_ctx* c, const StreamArgs& a, int variant) {
@@ -1149,10 +1154,11 @@ void launch_stream(regtopk_ctx* c, const StreamArgs& a, int variant) {
   k_stream<BF16, VEC><<<(unsigned)blocks, kStreamThreads, 0, c->stream>>>(a);
 }
 
-void post_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int N, int cluster, cudaStream_t s) {
+void post_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int N, int cluster, int threads,
+                 cudaStream_t s) {
   memset(cfg, 0, sizeof *cfg);
   cfg->gridDim = dim3((unsigned)(N * cluster), 1, 1);
-  cfg->blockDim = dim3(kBlockSel, 1, 1);
+  cfg->blockDim = dim3((unsigned)threads, 1, 1);
   cfg->dynamicSmemBytes = 0;
   cfg->stream = s;
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1173,7 +1179,7 @@ int choose_cluster(int N) {
   for (int cs = kMaxCluster; cs > 1; cs >>= 1) {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    post_config(&cfg, attr, N, cs, nullptr);
+    post_config(&cfg, attr, N, cs, kBlockPost, nullptr);
     int nclusters = 0;
     if (cudaOccupancyMaxActiveClusters(&nclusters, k_post, &cfg) != cudaSuccess) {
       cudaGetLastError();
@@ -1280,12 +1286,21 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   sa.grads = grads; sa.grad_ld = grad_ld; sa.eps = at<float>(c, L.off_eps); sa.ld = L.ld; sa.d = c->d;
   sa.k = c->k;
   sa.k_target = use_marks ? (2 * c->k < c->d ? 2 * c->k : c->d) : c->k;
-  sa.ctl = at<WorkerCtl>(c, L.off_ctl); sa.gctl = at<GlobalCtl>(c, L.off_gctl);
+  sa.ctl = at<WorkerCtl>(c, L.off_ctl);
+  sa.shist = at<u32>(c, L.off_shist);
   sa.ghist = at<u32>(c, L.off_ghist);
   sa.force_dense = (c->flags & REGTOPK_FLAG_FORCE_DENSE_SELECT) ? 1 : 0;
-  if (bf16) k_sample_cutoff<true><<<c->N, kBlockSel, sample_smem(), c->stream>>>(sa);
-  else k_sample_cutoff<false><<<c->N, kBlockSel, sample_smem(), c->stream>>>(sa);
-  if ((rc = after_launch(c))) return rc;
+  {
+    cudaLaunchConfig_t scfg;
+    cudaLaunchAttribute sattr[1];
+    post_config(&scfg, sattr, c->N, kSampleCluster, kBlockSel, c->stream);
+    scfg.dynamicSmemBytes = sample_smem();
+    cudaError_t se = bf16 ? cudaLaunchKernelEx(&scfg, k_sample_cutoff<true>, sa)
+                          : cudaLaunchKernelEx(&scfg, k_sample_cutoff<false>, sa);
+    c->launches++;
+    if (se != cudaSuccess) return note_cuda(c, se);
+    if ((rc = note_cuda(c, cudaGetLastError()))) return rc;
+  }
 
   StreamArgs st;
   st.grads = grads; st.grad_ld = grad_ld; st.eps = at<float>(c, L.off_eps); st.ld = L.ld; st.d = c->d;
@@ -1298,21 +1313,22 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   if ((rc = after_launch(c))) return rc;
 
   PostArgs pa;
-  pa.ctl = sa.ctl; pa.gctl = sa.gctl; pa.eps = at<float>(c, L.off_eps); pa.ld = L.ld; pa.d = c->d; pa.k = c->k;
+  pa.ctl = sa.ctl; pa.gctl = at<GlobalCtl>(c, L.off_gctl); pa.eps = at<float>(c, L.off_eps); pa.ld = L.ld; pa.d = c->d; pa.k = c->k;
   pa.g_prev = at<float>(c, L.off_g);
   pa.prev_idx = at<int32_t>(c, L.off_idx[prev]); pa.prev_val = at<float>(c, L.off_val[prev]);
   pa.omega = at<float>(c, L.off_omega); pa.mu = c->mu;
   pa.ovr_key = at<u32>(c, L.off_ovr_key); pa.ovr_comp = at<u64>(c, L.off_ovr_comp);
   pa.candA = at<u64>(c, L.off_candA); pa.candB = at<u64>(c, L.off_candB); pa.capA = L.capA; pa.stride = L.stride;
-  pa.ghist = at<u32>(c, L.off_ghist); pa.btot = at<u32>(c, L.off_btot);
+  pa.ghist = at<u32>(c, L.off_ghist); pa.shist = at<u32>(c, L.off_shist); pa.btot = at<u32>(c, L.off_btot);
   pa.mask_old = at<u32>(c, L.off_mask[prev]); pa.mask_new = at<u32>(c, L.off_mask[c->cur]);
-  pa.uprefix = at<u32>(c, L.off_uprefix); pa.W = L.W;
+  pa.qprefix = at<u32>(c, L.off_qprefix); pa.segtot = at<u32>(c, L.off_segtot);
+  pa.segbase = at<u32>(c, L.off_segbase); pa.W = L.W;
   pa.out_idx = out_idx; pa.out_val = out_val;
   pa.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); pa.cur_val = at<float>(c, L.off_val[c->cur]);
   pa.use_marks = use_marks; pa.has_stale = c->round >= 2;
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[1];
-  post_config(&cfg, attr, c->N, c->cluster, c->stream);
+  post_config(&cfg, attr, c->N, c->cluster, kBlockPost, c->stream);
   cudaError_t le = cudaLaunchKernelEx(&cfg, k_post, pa);
   c->launches++;
   if (le != cudaSuccess) return note_cuda(c, le);
@@ -1330,7 +1346,9 @@ int regtopk_aggregate(regtopk_ctx* c, float* out_g) {
   a.g = at<float>(c, L.off_g); a.N = c->N; a.k = c->k;
   a.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); a.cur_val = at<float>(c, L.off_val[c->cur]);
   a.prev_idx = at<int32_t>(c, L.off_idx[c->cur ^ 1]);
-  a.bitmask = at<u32>(c, L.off_mask[c->cur]); a.uprefix = at<u32>(c, L.off_uprefix); a.W = L.W;
+  a.bitmask = at<u32>(c, L.off_mask[c->cur]); a.qprefix = at<u32>(c, L.off_qprefix); a.segbase = at<u32>(c, L.off_segbase);
+  a.seg_units = ((L.W >> 3) + (int64_t)c->cluster * (kBlockPost / 32) - 1) / ((int64_t)c->cluster * (kBlockPost / 32));
+  a.W = L.W;
   a.omega = at<float>(c, L.off_omega);
   a.has_prev = c->round >= 1;
   const int64_t threads = (a.has_prev ? 2 : 1) * c->k * (int64_t)c->N;
@@ -1404,6 +1422,7 @@ int regtopk_get_stats(regtopk_ctx* c, regtopk_stats* out) {
     out->candidates_last = 0;
     for (int n = 0; n < c->N; ++n) out->candidates_last += w[n].cand_count;
     out->candidate_capacity = c->L.capA;
+    out->device_error_bits = (int64_t)h.err;
   }
   free(w);
   return rc;

@@ -122,10 +122,13 @@ def test_forced_dense_select(mu):
                expect_dense=True)
 
 
+SAMPLE_SECTORS = 8192  # 32-byte sectors the library's cutoff sample reads per worker
+
+
 def _sample_positions(d):
     Q = (d + 7) // 8
-    s = np.arange(4096, dtype=np.int64)
-    q = s * Q // 4096
+    s = np.arange(SAMPLE_SECTORS, dtype=np.int64)
+    q = s * Q // SAMPLE_SECTORS
     return (q[:, None] * 8 + np.arange(8)[None, :]).reshape(-1)
 
 
