@@ -144,18 +144,6 @@ __device__ __forceinline__ void block_find_from_top(const u32* hist, int nbins, 
   __syncthreads();
 }
 
-// Warp-aggregated reservation in a shared counter: returns this lane's slot if pred, any value if not.
-__device__ __forceinline__ u32 warp_reserve(bool pred, u32* s_counter) {
-  const u32 m = __ballot_sync(kFull, pred);
-  if (m == 0) return 0;
-  const int lane = threadIdx.x & 31;
-  const int leader = __ffs(m) - 1;
-  u32 base = 0;
-  if (lane == leader) base = atomicAdd(s_counter, (u32)__popc(m));
-  base = __shfl_sync(kFull, base, leader);
-  return base + (u32)__popc(m & ((1u << lane) - 1u));
-}
-
 // ---------------------------------------------------------------------------------------------
 // tanh(x), x >= 0, as a fixed sequence of individually rounded binary32 operations:
 //   x >= 9.25 -> 1;   x < 0.25 -> x + x*q with the odd Taylor terms up to x^9;
@@ -208,6 +196,8 @@ constexpr int kSampleCluster = 8;
 constexpr int kSamplePerBlock = kSampleMax / kSampleCluster;  // 8192: eight per thread
 constexpr int kSampleBins = 16384;
 constexpr int kSampleShift = 17;  // key >> 17: sign-less exponent and six mantissa bits
+constexpr int kSamplePadded = kSampleBins + kSampleBins / 16;
+__device__ __forceinline__ u32 sample_slot(u32 bin) { return bin + (bin >> 4); }
 
 struct SampleArgs {
   const void* grads;
@@ -233,7 +223,7 @@ __device__ __forceinline__ void flush_hist(const u32* s_hist, u32* g_hist, int n
 
 template <bool BF16>
 __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
-  extern __shared__ u32 s_hist[];  // kSampleBins
+  extern __shared__ u32 s_hist[];  // kSampleBins bins, one pad word after every 16 (bank-conflict-free per-thread runs)
   __shared__ u32 s_scan[33];
   __shared__ u32 s_res[3];
   cg::cluster_group cl = cg::this_cluster();
@@ -278,17 +268,20 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
       e[u] = ok[u] ? eps_row[j] : 0.0f;
       g[u] = ok[u] ? load_grad<BF16>(grow, j) : 0.0f;
     }
-    for (int i = tid; i < kSampleBins; i += blockDim.x) s_hist[i] = 0;  // while the loads are in flight
+    for (int i = tid; i < kSamplePadded; i += blockDim.x) s_hist[i] = 0;  // while the loads are in flight
     __syncthreads();
 #pragma unroll
     for (int u = 0; u < 8; ++u)
-      if (ok[u]) atomicAdd(&s_hist[(__float_as_uint(__fadd_rn(e[u], g[u])) & 0x7FFFFFFFu) >> kSampleShift], 1u);
+      if (ok[u]) atomicAdd(&s_hist[sample_slot((__float_as_uint(__fadd_rn(e[u], g[u])) & 0x7FFFFFFFu) >> kSampleShift)], 1u);
   }
   __syncthreads();
-  flush_hist(s_hist, shist, kSampleBins);
+  for (int i = tid; i < kSampleBins; i += blockDim.x) {
+    const u32 v = s_hist[sample_slot((u32)i)];
+    if (v) atomicAdd(&shist[i], v);
+  }
   cl.sync();  // histogram of the whole sample complete
   if (rk != 0) return;
-  for (int i = tid; i < kSampleBins; i += blockDim.x) s_hist[i] = __ldcg(&shist[i]);
+  for (int i = tid; i < kSampleBins; i += blockDim.x) s_hist[sample_slot((u32)i)] = __ldcg(&shist[i]);
   __syncthreads();
 
   // Ranks to read off the sample.  The number of sample points above a quantile is close to Poisson
@@ -301,18 +294,37 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
   const u32 r_lo = r_lo_d > (double)M ? (u32)M + 1u : (u32)r_lo_d;
   const u32 r_hi = r_hi_d < 1.0 ? 1u : (u32)r_hi_d;
 
+  // One suffix scan serves both ranks.  A thread owns 16 consecutive bins, counted from the top.
+  constexpr int kPer = kSampleBins / kBlockSel;
+  u32 mine[kPer];
+  u32 sum = 0;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    mine[i] = s_hist[sample_slot((u32)(kSampleBins - 1 - (tid * kPer + i)))];
+    sum += mine[i];
+  }
+  if (tid == 0) { s_res[0] = kFull; s_res[1] = kFull; }
+  u32 total;
+  const u32 excl = block_excl_scan(sum, s_scan, &total);
+  const u32 want[2] = {r_hi, r_lo};
+#pragma unroll
+  for (int w = 0; w < 2; ++w) {
+    if (excl < want[w] && want[w] <= excl + sum) {
+      u32 acc = excl;
+#pragma unroll
+      for (int i = 0; i < kPer; ++i) {
+        if (acc < want[w] && want[w] <= acc + mine[i]) s_res[w] = (u32)(kSampleBins - 1 - (tid * kPer + i));
+        acc += mine[i];
+      }
+    }
+  }
+  __syncthreads();
   // upper end of the key range the select should resolve finely: the k-th largest score cannot
   // exceed the k-th largest |a|, estimated from above by the sample's r_hi-th largest
-  block_find_from_top(s_hist, kSampleBins, r_hi, s_scan, s_res);
   u32 hi_key = s_res[0] == kFull ? 0x7F7FFFFFu : (((s_res[0] + 1u) << kSampleShift) - 1u);
-  __syncthreads();
   if (r_hi_d < 1.0) hi_key = hi_key < 0x7F000000u ? hi_key + (1u << 23) : 0x7F7FFFFFu;  // an octave of slack
-
-  u32 cutoff = 0;  // lower edge of the bin that holds the r_lo-th largest sample
-  if (r_lo <= (u32)M) {
-    block_find_from_top(s_hist, kSampleBins, r_lo, s_scan, s_res);
-    if (s_res[0] != kFull) cutoff = s_res[0] << kSampleShift;
-  }
+  // the cutoff: lower edge of the bin that holds the r_lo-th largest sample (0: keep everything)
+  const u32 cutoff = (r_lo <= (u32)M && s_res[1] != kFull) ? s_res[1] << kSampleShift : 0u;
   if (tid == 0) {
     const u32 range = hi_key > cutoff ? hi_key - cutoff : 0u;
     u32 shift = 0;
@@ -1138,7 +1150,7 @@ int after_launch(regtopk_ctx* c) {
   return note_cuda(c, cudaGetLastError());
 }
 
-size_t sample_smem() { return (size_t)kSampleBins * sizeof(u32); }
+size_t sample_smem() { return (size_t)kSamplePadded * sizeof(u32); }
 
 template <bool BF16, bool VEC>
 void launch_stream(regtopk_ctx* c, const StreamArgs& a, int variant) {
