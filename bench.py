@@ -195,7 +195,8 @@ def main():
     ring_n = args.ring or w.steps
     ring_n = int(max(2, min(ring_n, (free * 0.5) // per_batch)))
     ring = [stream.next() for _ in range(ring_n)]
-    lib = pkg.RegTopK(w.d, w.N, k, mu=w.mu, grad_dtype=tdt, flags=binding.FLAG_HOST_STAGING)
+    lib = pkg.RegTopK(w.d, w.N, k, mu=w.mu, grad_dtype=tdt,
+                      flags=binding.FLAG_HOST_STAGING if args.e2e_steps > 0 else 0)
     out_idx = torch.empty((w.N, k), dtype=torch.int32, device=dev)
     out_val = torch.empty((w.N, k), dtype=torch.float32, device=dev)
 
@@ -242,18 +243,20 @@ def main():
     kern_ms, calls = lib.profile_read()
     lib.profile_enable(False)
     # ---- end to end through host buffers ----
-    h_g = [ring[i].cpu().pin_memory() for i in range(min(2, ring_n))]
-    h_idx = torch.empty((w.N, k), dtype=torch.int32).pin_memory()
-    h_val = torch.empty((w.N, k), dtype=torch.float32).pin_memory()
-    h_agg = torch.empty(w.d, dtype=torch.float32).pin_memory()
-    for i in range(2):
-        lib.round_host(h_g[i % len(h_g)], h_idx, h_val, h_agg)
-    barrier()
-    t0 = time.perf_counter()
-    for i in range(args.e2e_steps):
-        lib.round_host(h_g[i % len(h_g)], h_idx, h_val, h_agg)  # synchronises each step
-    barrier()
-    e2e_s = time.perf_counter() - t0
+    e2e_s = float("nan")
+    if args.e2e_steps > 0:
+        h_g = [ring[i].cpu().pin_memory() for i in range(min(2, ring_n))]
+        h_idx = torch.empty((w.N, k), dtype=torch.int32).pin_memory()
+        h_val = torch.empty((w.N, k), dtype=torch.float32).pin_memory()
+        h_agg = torch.empty(w.d, dtype=torch.float32).pin_memory()
+        for i in range(2):
+            lib.round_host(h_g[i % len(h_g)], h_idx, h_val, h_agg)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(args.e2e_steps):
+            lib.round_host(h_g[i % len(h_g)], h_idx, h_val, h_agg)  # synchronises each step
+        barrier()
+        e2e_s = time.perf_counter() - t0
     lib.status()
     stats_end = lib.stats()
 
@@ -282,7 +285,7 @@ def main():
                        "candidates_last": stats_end["candidates_last"],
                        "ms_per_step_with_kernel_events": ms_prof / nprof},
             "clocks": clocks,
-            "e2e": {"value": world * coords * args.e2e_steps / e2e_all / 1e9, "unit": UNIT,
+            "e2e": {"value": (world * coords * args.e2e_steps / e2e_all / 1e9) if args.e2e_steps > 0 else None, "unit": UNIT,
                     "h2d_bytes_per_step": w.N * stream.ld * bpe, "d2h_bytes_per_step": 2 * w.N * k * 4 + w.d * 4},
             "gpu_launches": launches,
             "roofline": {"bound": "hbm", "kernel": "k_stream", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -290,7 +293,7 @@ def main():
                          "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": kern_avg_ms},
         }
         if world == 1 and not args.no_cpu_baseline:
-            del ring, h_g
+            del ring
             torch.cuda.empty_cache()
             line["cpu_baseline"] = cpu_baseline(w, k, args.seed)
         print(json.dumps(line), flush=True)

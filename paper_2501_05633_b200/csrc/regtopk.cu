@@ -303,6 +303,7 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
     mine[i] = s_hist[sample_slot((u32)(kSampleBins - 1 - (tid * kPer + i)))];
     sum += mine[i];
   }
+  __shared__ u32 s_frac[2];  // for the r_lo bin: sample points in it, and how many of them rank at or above r_lo
   if (tid == 0) { s_res[0] = kFull; s_res[1] = kFull; }
   u32 total;
   const u32 excl = block_excl_scan(sum, s_scan, &total);
@@ -313,7 +314,10 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
       u32 acc = excl;
 #pragma unroll
       for (int i = 0; i < kPer; ++i) {
-        if (acc < want[w] && want[w] <= acc + mine[i]) s_res[w] = (u32)(kSampleBins - 1 - (tid * kPer + i));
+        if (acc < want[w] && want[w] <= acc + mine[i]) {
+          s_res[w] = (u32)(kSampleBins - 1 - (tid * kPer + i));
+          if (w == 1) { s_frac[0] = mine[i]; s_frac[1] = want[w] - acc; }
+        }
         acc += mine[i];
       }
     }
@@ -323,8 +327,15 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
   // exceed the k-th largest |a|, estimated from above by the sample's r_hi-th largest
   u32 hi_key = s_res[0] == kFull ? 0x7F7FFFFFu : (((s_res[0] + 1u) << kSampleShift) - 1u);
   if (r_hi_d < 1.0) hi_key = hi_key < 0x7F000000u ? hi_key + (1u << 23) : 0x7F7FFFFFu;  // an octave of slack
-  // the cutoff: lower edge of the bin that holds the r_lo-th largest sample (0: keep everything)
-  const u32 cutoff = (r_lo <= (u32)M && s_res[1] != kFull) ? s_res[1] << kSampleShift : 0u;
+  // the cutoff: inside the bin that holds the r_lo-th largest sample, placed as if the bin's sample
+  // points were spread evenly over it (0: keep everything).  Error feedback piles entries up just
+  // below the selection threshold, so a cutoff a whole bin too low would gather far too many.
+  u32 cutoff = 0u;
+  if (r_lo <= (u32)M && s_res[1] != kFull) {
+    const u32 width = 1u << kSampleShift;
+    const u32 below = (u32)(((u64)(s_frac[0] - s_frac[1]) * width) / (s_frac[0] + 1u));  // offset from the bin's lower edge
+    cutoff = (s_res[1] << kSampleShift) + below;
+  }
   if (tid == 0) {
     const u32 range = hi_key > cutoff ? hi_key - cutoff : 0u;
     u32 shift = 0;
@@ -1068,7 +1079,7 @@ Layout make_layout(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
   L.W = (int64_t)align_up((size_t)((d + 31) / 32), 32);
   const int64_t M = d < kSampleMax ? d : kSampleMax;
   const int64_t kt = pr->mu > 0.0f ? (2 * k < d ? 2 * k : d) : k;
-  int64_t cap = 2 * kt + 64 * ((d + M - 1) / M) + 4096;
+  int64_t cap = 3 * kt + 64 * ((d + M - 1) / M) + 4096;
   if (cap > d) cap = d;
   if (cap < k) cap = k;
   L.capA = cap;
