@@ -211,6 +211,17 @@ struct SampleArgs {
   u32* ghist;  // [N][4][kBins] histograms of k_post, cleared here
   u32* shist;  // [N][kSampleBins] histogram of this kernel; zero on entry (k_post clears it again)
   int force_dense;
+  // Clusters beyond the first N compute the regularised scores of the previous support
+  // (Eq. (Delta_def), Algorithm 2 steps 8-9) while the first N sample.  On that support the
+  // residual is +0, so the accumulator there is 0 + g.
+  int N;
+  int use_marks;
+  const float* g_prev;
+  const int32_t* prev_idx;  // [N][k]
+  const float* prev_val;    // [N][k]
+  const float* omega;
+  float mu;
+  u32* ovr_key;             // [N][k] out: score bits
 };
 
 // Add a block's histogram to the cluster's in global memory (non-empty bins only).
@@ -230,6 +241,49 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
   const u32 rk = cl.block_rank();
   const int n = blockIdx.x / kSampleCluster;
   const int tid = threadIdx.x;
+  if (n >= p.N) {  // an override cluster: no barriers on this path
+    if (!p.use_marks) return;
+    const int64_t total = p.k * p.N;
+    const int64_t nthreads = (int64_t)(gridDim.x - p.N * kSampleCluster) * blockDim.x;
+    const int64_t first = (int64_t)(blockIdx.x - p.N * kSampleCluster) * blockDim.x + tid;
+    for (int64_t t0 = first; t0 < total; t0 += 4 * nthreads) {
+      int32_t j[4];
+      float ap[4], G[4], gr[4];
+      int wn[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int64_t t = t0 + q * nthreads;
+        const bool in = t < total;
+        j[q] = in ? p.prev_idx[t] : 0;
+        ap[q] = in ? p.prev_val[t] : 0.0f;
+        wn[q] = in ? (int)(t / p.k) : 0;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const bool in = t0 + q * nthreads < total;
+        G[q] = in ? p.g_prev[j[q]] : 0.0f;
+        gr[q] = in ? load_grad<BF16>(static_cast<const char*>(p.grads) + (size_t)wn[q] * p.grad_ld * (BF16 ? 2 : 4), j[q]) : 0.0f;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int64_t t = t0 + q * nthreads;
+        if (t < total) {
+          const float w = p.omega[wn[q]];
+          const float a = __fadd_rn(0.0f, gr[q]);
+          const float num = __fsub_rn(G[q], __fmul_rn(w, ap[q]));
+          const float den = __fmul_rn(w, a);
+          float m = 1.0f;
+          if (den != 0.0f) {
+            const float delta = __fdiv_rn(num, den);
+            const float r = fabsf(__fadd_rn(1.0f, delta));
+            m = tanh_fixed(__fdiv_rn(r, p.mu));
+          }
+          p.ovr_key[t] = __float_as_uint(__fmul_rn(fabsf(a), m));
+        }
+      }
+    }
+    return;
+  }
   WorkerCtl* ctl = p.ctl + n;
   u32* shist = p.shist + (size_t)n * kSampleBins;
 
@@ -366,18 +420,51 @@ struct StreamArgs {
   u64* cand;       // [N][stride]
   int64_t cap;     // entries of a row the stream pass may fill
   int64_t stride;
+  const u32* marks;  // [N][W] last round's mask, or NULL: entries on it are not candidates (their
+  int64_t W;         // regularised score comes from the override list instead)
 };
 
+// Write a warp's staged hits to the worker's candidate list.  With a previous mask, the entries on it
+// are dropped first: the probes of a flush are issued four per lane at a time, so the warp waits for
+// memory a few times per flush, not once per hit.
 __device__ __forceinline__ void stream_flush(u64* list, u32& wcount, WorkerCtl* ctl, u64* cand,
-                                             int64_t cap, int lane) {
+                                             int64_t cap, const u32* marks, int lane) {
   __syncwarp();
   if (wcount) {
-    u32 base = 0;
-    if (lane == 0) base = atomicAdd(&ctl->cand_count, wcount);
-    base = __shfl_sync(kFull, base, 0);
-    for (u32 i = lane; i < wcount; i += 32) {
-      const u64 pos = (u64)base + i;
-      if (pos < (u64)cap) cand[pos] = list[i];
+    if (marks) {
+      u32 kept = 0;
+      const u32 total = wcount;
+#pragma unroll 1
+      for (u32 r0 = 0; r0 < total; r0 += 128) {
+        u64 ent[4];
+        u32 word[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const u32 i = r0 + (u32)r * 32 + lane;
+          ent[r] = i < total ? list[i] : 0ull;
+          word[r] = i < total ? __ldg(&marks[composite_idx(ent[r]) >> 5]) : 0u;
+        }
+        __syncwarp();  // every lane has read its entries before any is overwritten
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const u32 i = r0 + (u32)r * 32 + lane;
+          const bool keep = i < total && !((word[r] >> (composite_idx(ent[r]) & 31)) & 1u);
+          const u32 m = __ballot_sync(kFull, keep);
+          if (keep) list[kept + __popc(m & ((1u << lane) - 1u))] = ent[r];  // kept <= r0 + 32 r: behind the reads
+          kept += __popc(m);
+        }
+        __syncwarp();
+      }
+      wcount = kept;
+    }
+    if (wcount) {
+      u32 base = 0;
+      if (lane == 0) base = atomicAdd(&ctl->cand_count, wcount);
+      base = __shfl_sync(kFull, base, 0);
+      for (u32 i = lane; i < wcount; i += 32) {
+        const u64 pos = (u64)base + i;
+        if (pos < (u64)cap) cand[pos] = list[i];
+      }
     }
   }
   wcount = 0;
@@ -385,7 +472,7 @@ __device__ __forceinline__ void stream_flush(u64* list, u32& wcount, WorkerCtl* 
 }
 
 template <bool BF16, bool VEC>
-__global__ void __launch_bounds__(kStreamThreads) k_stream(StreamArgs p) {
+__global__ void __launch_bounds__(kStreamThreads, 3) k_stream(StreamArgs p) {
   __shared__ u64 s_list[kStreamThreads / 32][kWarpList];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   u64* list = s_list[warp];
@@ -402,7 +489,8 @@ __global__ void __launch_bounds__(kStreamThreads) k_stream(StreamArgs p) {
     const int n = (int)(c / chunks_per_row);
     const int64_t base = (c - (int64_t)n * chunks_per_row) << 9;
     if (n != cur_n) {
-      if (cur_n >= 0) stream_flush(list, wcount, p.ctl + cur_n, p.cand + (size_t)cur_n * p.stride, p.cap, lane);
+      if (cur_n >= 0) stream_flush(list, wcount, p.ctl + cur_n, p.cand + (size_t)cur_n * p.stride, p.cap,
+                                  p.marks ? p.marks + (size_t)cur_n * p.W : nullptr, lane);
       cur_n = n;
       cutoff = p.ctl[n].cutoff;
       eps_row = p.eps + (size_t)n * p.ld;
@@ -462,11 +550,13 @@ __global__ void __launch_bounds__(kStreamThreads) k_stream(StreamArgs p) {
         if (h3) list[wcount + __popc(m & lt)] = make_composite(k3, (u32)j + 3);
         wcount += __popc(m);
         if (wcount >= kWarpList - 128)  // the next step adds at most 128
-          stream_flush(list, wcount, p.ctl + cur_n, p.cand + (size_t)cur_n * p.stride, p.cap, lane);
+          stream_flush(list, wcount, p.ctl + cur_n, p.cand + (size_t)cur_n * p.stride, p.cap,
+                                  p.marks ? p.marks + (size_t)cur_n * p.W : nullptr, lane);
       }
     }
   }
-  if (cur_n >= 0) stream_flush(list, wcount, p.ctl + cur_n, p.cand + (size_t)cur_n * p.stride, p.cap, lane);
+  if (cur_n >= 0) stream_flush(list, wcount, p.ctl + cur_n, p.cand + (size_t)cur_n * p.stride, p.cap,
+                                  p.marks ? p.marks + (size_t)cur_n * p.W : nullptr, lane);
 }
 
 
@@ -648,8 +738,6 @@ __global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
   u64* O = p.ovr_comp + (size_t)n * p.k;
   u32* okey = p.ovr_key + (size_t)n * p.k;
   const int32_t* prev_idx = p.prev_idx + (size_t)n * p.k;
-  const float* prev_val = p.prev_val + (size_t)n * p.k;
-  const u32* mask_old = p.mask_old + (size_t)n * p.W;
   u32* mask = p.mask_new + (size_t)n * p.W;
   u32* ghist = p.ghist + (size_t)n * 4 * kBins;
   u32* btot = p.btot + (size_t)n * 2 * kMaxCluster;
@@ -671,62 +759,37 @@ __global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
   for (int i = tid; i < kBins; i += blockDim.x) sh.hist[i] = 0;
   for (u32 i = first_t; i < (u32)kSampleBins; i += stride_t) p.shist[(size_t)n * kSampleBins + i] = 0;
   __syncthreads();
-  // ---- one fused sweep, so that the independent loads of its three jobs are in flight together:
+  // ---- one sweep over the lists, a single wave of coalesced loads per step:
   //   (a) the mask buffer of this round still holds the mask of two rounds ago: clear those words;
-  //   (b) regularised scores on the previous support (Eq. (Delta_def), Algorithm 2 step 9);
-  //   (c) filter and histogram the candidates: those on the previous support are dropped (their
-  //       score is the override's); a thread meets the same items again in the classify pass ----
+  //   (b) the override scores (written by k_sample_cutoff's override clusters) that reach the
+  //       cutoff become composites and enter the histogram;
+  //   (c) the candidates (k_stream already dropped those on the previous support) enter it too ----
   {
-    const float w = p.omega[n];
     const u32 span = !dense && ncand > k ? ncand : k;
-    constexpr int kP0 = 4;  // items per thread in flight
+    constexpr int kP0 = 8;  // items per thread in flight
     for (u32 i0 = first_t; i0 < span; i0 += kP0 * stride_t) {
-      bool in_k[kP0], do_ovr[kP0], do_cand[kP0];
       int32_t stale[kP0], j[kP0];
-      float ap[kP0], a[kP0], G[kP0];
+      u32 key[kP0];
       u64 c[kP0];
-      u32 mword[kP0];
 #pragma unroll
-      for (int q = 0; q < kP0; ++q) {  // first wave of loads
+      for (int q = 0; q < kP0; ++q) {
         const u32 i = i0 + q * stride_t;
-        in_k[q] = i < k;
-        do_ovr[q] = in_k[q] && p.use_marks;
-        do_cand[q] = !dense && i < ncand;
-        stale[q] = (in_k[q] && p.has_stale) ? p.cur_idx[obase + i] : 0;
-        j[q] = do_ovr[q] ? prev_idx[i] : 0;
-        ap[q] = do_ovr[q] ? prev_val[i] : 0.0f;
-        c[q] = do_cand[q] ? A[i] : 0ull;
-      }
-#pragma unroll
-      for (int q = 0; q < kP0; ++q) {  // second wave, dependent on the first
-        a[q] = do_ovr[q] ? eps_row[j[q]] : 0.0f;
-        G[q] = do_ovr[q] ? p.g_prev[j[q]] : 0.0f;
-        mword[q] = (do_cand[q] && p.use_marks) ? mask_old[composite_idx(c[q]) >> 5] : 0u;
+        const bool in_k = i < k;
+        stale[q] = (in_k && p.has_stale) ? p.cur_idx[obase + i] : -1;
+        j[q] = (in_k && p.use_marks) ? prev_idx[i] : -1;
+        key[q] = (in_k && p.use_marks) ? okey[i] : 0u;
+        c[q] = (!dense && i < ncand) ? A[i] : 0ull;
       }
 #pragma unroll
       for (int q = 0; q < kP0; ++q) {
         const u32 i = i0 + q * stride_t;
-        if (in_k[q] && p.has_stale) mask[(u32)stale[q] >> 5] = 0u;
-        if (do_ovr[q]) {
-          const float num = __fsub_rn(G[q], __fmul_rn(w, ap[q]));
-          const float den = __fmul_rn(w, a[q]);
-          float m = 1.0f;
-          if (den != 0.0f) {
-            const float delta = __fdiv_rn(num, den);
-            const float r = fabsf(__fadd_rn(1.0f, delta));
-            m = tanh_fixed(__fdiv_rn(r, p.mu));
-          }
-          const u32 key = __float_as_uint(__fmul_rn(fabsf(a[q]), m));
-          const u64 oc = key >= cutoff ? make_composite(key, (u32)j[q]) : 0ull;
-          okey[i] = key;
+        if (stale[q] >= 0) mask[(u32)stale[q] >> 5] = 0u;
+        if (j[q] >= 0) {
+          const u64 oc = key[q] >= cutoff ? make_composite(key[q], (u32)j[q]) : 0ull;
           O[i] = oc;
-          if (!dense && oc) atomicAdd(&sh.hist[select_bin(key, cutoff, bshift)], 1u);
+          if (!dense && oc) atomicAdd(&sh.hist[select_bin(key[q], cutoff, bshift)], 1u);
         }
-        if (do_cand[q]) {
-          const u32 cidx = composite_idx(c[q]);
-          if ((mword[q] >> (cidx & 31)) & 1u) A[i] = 0ull;
-          else atomicAdd(&sh.hist[select_bin((u32)(c[q] >> 32), cutoff, bshift)], 1u);
-        }
+        if (c[q]) atomicAdd(&sh.hist[select_bin((u32)(c[q] >> 32), cutoff, bshift)], 1u);
       }
     }
   }
@@ -908,7 +971,8 @@ __global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
     }
   }
   for (int part = 0; part < 2; ++part) {
-    // normal path: candidates, then overrides; dense path: its k winners, nothing else
+    // normal path: candidates, then overrides; dense path: its k winners, nothing else.  Items
+    // below the threshold bin cannot have won and are skipped without touching memory.
     const u64* items = part == 0 ? A : O;
     const u32 count = part == 0 ? (took_dense ? k : ncand) : (took_dense ? 0u : novr);
     for (u32 i0 = first_t; i0 < count; i0 += 4 * stride_t) {
@@ -916,6 +980,7 @@ __global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
       uint4 qw[4];
       u32 qp[4];
       float vv[4];
+      bool live[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const u32 i = i0 + q * stride_t;
@@ -924,14 +989,14 @@ __global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const u32 idx = composite_idx(c[q]);
-        const bool valid = c[q] != 0ull;
-        qw[q] = valid ? __ldcg(quads + (idx >> 7)) : make_uint4(0, 0, 0, 0);
-        qp[q] = valid ? __ldcg(qpre + (idx >> 7)) : 0u;
-        vv[q] = valid ? eps_row[idx] : 0.0f;  // fetched before the bit test: most candidates near the top win
+        live[q] = c[q] != 0ull && (took_dense || select_bin((u32)(c[q] >> 32), cutoff, bshift) >= b1);
+        qw[q] = live[q] ? __ldcg(quads + (idx >> 7)) : make_uint4(0, 0, 0, 0);
+        qp[q] = live[q] ? __ldcg(qpre + (idx >> 7)) : 0u;
+        vv[q] = live[q] ? eps_row[idx] : 0.0f;
       }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        if (c[q] == 0ull) continue;
+        if (!live[q]) continue;
         const u32 idx = composite_idx(c[q]);
         const u32 w[4] = {qw[q].x, qw[q].y, qw[q].z, qw[q].w};
         const u32 wsel = (idx >> 5) & 3u;
@@ -1312,11 +1377,16 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   sa.ctl = at<WorkerCtl>(c, L.off_ctl);
   sa.shist = at<u32>(c, L.off_shist);
   sa.ghist = at<u32>(c, L.off_ghist);
+  sa.N = c->N; sa.use_marks = use_marks; sa.g_prev = at<float>(c, L.off_g);
+  sa.prev_idx = at<int32_t>(c, L.off_idx[prev]); sa.prev_val = at<float>(c, L.off_val[prev]);
+  sa.omega = at<float>(c, L.off_omega); sa.mu = c->mu; sa.ovr_key = at<u32>(c, L.off_ovr_key);
   sa.force_dense = (c->flags & REGTOPK_FLAG_FORCE_DENSE_SELECT) ? 1 : 0;
   {
     cudaLaunchConfig_t scfg;
     cudaLaunchAttribute sattr[1];
-    post_config(&scfg, sattr, c->N, kSampleCluster, kBlockSel, c->stream);
+    int extra = use_marks ? (c->num_sms - c->N * kSampleCluster) / kSampleCluster : 0;  // override clusters
+    if (use_marks && extra < 1) extra = 1;
+    post_config(&scfg, sattr, c->N + extra, kSampleCluster, kBlockSel, c->stream);
     scfg.dynamicSmemBytes = sample_smem();
     cudaError_t se = bf16 ? cudaLaunchKernelEx(&scfg, k_sample_cutoff<true>, sa)
                           : cudaLaunchKernelEx(&scfg, k_sample_cutoff<false>, sa);
@@ -1328,6 +1398,7 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   StreamArgs st;
   st.grads = grads; st.grad_ld = grad_ld; st.eps = at<float>(c, L.off_eps); st.ld = L.ld; st.d = c->d;
   st.N = c->N; st.ctl = sa.ctl; st.cand = at<u64>(c, L.off_candA); st.cap = L.capA; st.stride = L.stride;
+  st.marks = use_marks ? at<u32>(c, L.off_mask[prev]) : nullptr; st.W = L.W;
   const bool prof = c->profiling && c->n_events < kMaxProfile;
   if (prof) cudaEventRecord(c->ev0[c->n_events], c->stream);
   if (bf16) { if (vec) launch_stream<true, true>(c, st, 3); else launch_stream<true, false>(c, st, 2); }
