@@ -95,6 +95,21 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def workload_label(w, k, sparsity):
+    return (f"{w.name}-shaped gradient d={w.d} N={w.N} k={k} ({sparsity:g} of d) mu={w.mu} "
+            f"grads={w.grad_dtype}")
+
+
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the time)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
 def run_reference(args, rank, world):
     """The CPU oracle, as it stands, on a bounded sample of the workload (rank 0 only)."""
     if rank != 0:
@@ -106,14 +121,14 @@ def run_reference(args, rank, world):
     w = synth.workload(args.workload)
     s = w.sparsity[args.sparsity_index]
     total_steps = args.steps + args.warmup
-    budget = 150.0 / max(1, total_steps)  # seconds of oracle work per step
+    budget = min(4.0, 150.0 / max(1, total_steps))  # seconds of oracle work per step
     # calibrate the oracle's rate on a small slice
     dcal = 200_000
     wc = synth.workload(args.workload, scale_to=dcal)
     gs = synth.GradientStream(wc, device="cpu", seed=args.seed)
     o = OracleRegTopK(wc.d, 1, max(1, int(s * wc.d + 0.5)), w.mu)
     g = gs.next()[:1]
-    from tests.parity import to_oracle_view
+    from oracle.oracle import grads_view as to_oracle_view
     t0 = time.perf_counter()
     o.worker_step(to_oracle_view(g, wc.d)); o.aggregate()
     rate = wc.d / (time.perf_counter() - t0)
@@ -138,7 +153,7 @@ def run_reference(args, rank, world):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": el / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{w.name} d={w.d} N={w.N} k={int(s * w.d + 0.5)} mu={w.mu}", "sample": sample},
+            "config": {"workload": workload_label(w, int(s * w.d + 0.5), s), "sample": sample},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -150,7 +165,7 @@ def cpu_baseline(w, k, seed):
     import torch
     from paper_2501_05633_b200 import synth
     from oracle.oracle import OracleRegTopK
-    from tests.parity import to_oracle_view
+    from oracle.oracle import grads_view as to_oracle_view
     nw = min(w.N, 4)  # bounded: a full sort of d entries per worker costs about a second per 10M
     wsamp = synth.workload(w.name)
     wsamp.N = nw
@@ -260,10 +275,7 @@ def main():
     lib.status()
     stats_end = lib.stats()
 
-    t_max = torch.tensor([ms, e2e_s], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_max, op=dist.ReduceOp.MAX)
-    ms_all, e2e_all = float(t_max[0]), float(t_max[1])
+    ms_all, e2e_all = max_over_ranks([ms, e2e_s], dev, world)
     if rank == 0:
         coords = w.N * w.d
         value = world * coords * args.steps / (ms_all * 1e-3) / 1e9
@@ -276,7 +288,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_all / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{w.name}-shaped gradient d={w.d} N={w.N} k={k} ({w.sparsity[args.sparsity_index]:g} of d) mu={w.mu} grads={w.grad_dtype}",
+            "config": {"workload": workload_label(w, k, w.sparsity[args.sparsity_index]),
                        "replicas": world, "parallelism": "replicas only (the path runs on one GPU)",
                        "l2": f"inputs larger than L2 ({per_batch / 1e6:.0f} MB per step, ring of {ring_n} batches)",
                        "step_hbm_gbs": step_gbs, "step_frac_of_measured_peak": step_gbs / peak,

@@ -141,6 +141,14 @@ def default() -> OracleAPI:
     return _default
 
 
+def grads_view(grads_cpu, d: int) -> np.ndarray:
+    """[N, ld] torch CPU tensor -> [N, d] numpy array the oracle reads (bfloat16 as uint16 bit patterns)."""
+    import torch
+    if grads_cpu.dtype == torch.bfloat16:
+        return np.ascontiguousarray(grads_cpu.view(torch.int16).numpy().view(np.uint16)[:, :d])
+    return np.ascontiguousarray(grads_cpu.numpy()[:, :d])
+
+
 class OracleRegTopK:
     """State of N workers and the server across rounds (Algorithm 2's initialisation and loop).
 

@@ -3,15 +3,11 @@ seeded inputs.  Index sets, sent values, residuals and the aggregate must agree 
 import numpy as np
 import torch
 
-from oracle.oracle import OracleRegTopK
+from oracle.oracle import OracleRegTopK, grads_view
 from paper_2501_05633_b200 import RegTopK
 
 
-def to_oracle_view(grads_cpu: torch.Tensor, d: int) -> np.ndarray:
-    """[N, ld] torch CPU tensor -> [N, d] numpy array the oracle reads (bf16 as uint16 bit patterns)."""
-    if grads_cpu.dtype == torch.bfloat16:
-        return np.ascontiguousarray(grads_cpu.view(torch.int16).numpy().view(np.uint16)[:, :d])
-    return np.ascontiguousarray(grads_cpu.numpy()[:, :d])
+to_oracle_view = grads_view
 
 
 def bits(x):
