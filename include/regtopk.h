@@ -42,7 +42,8 @@ enum {
   REGTOPK_ERR_SEQUENCE = -3,            /* worker_step twice without aggregate, or aggregate first     */
   REGTOPK_ERR_CUDA = -4,                /* a CUDA runtime call or launch failed                        */
   REGTOPK_ERR_INTERNAL = -5,            /* the device reported an inconsistent selection (a bug)       */
-  REGTOPK_ERR_NO_DEVICE = -6            /* no usable sm_100 device / kernel image                      */
+  REGTOPK_ERR_NO_DEVICE = -6,           /* no usable sm_100 device / kernel image                      */
+  REGTOPK_ERR_TOO_LARGE = -7            /* the problem exceeds a fixed built-in capacity               */
 };
 
 enum { REGTOPK_GRAD_F32 = 0, REGTOPK_GRAD_BF16 = 1 };
@@ -133,6 +134,30 @@ int regtopk_profile_read(regtopk_ctx* ctx, double* stream_kernel_ms, int64_t* ca
 
 /* Test introspection: device pointer to the residuals eps ([N][*ld] binary32, *ld >= d). */
 int regtopk_debug_residual(regtopk_ctx* ctx, const float** dev_ptr, int64_t* ld);
+
+/* Server aggregation from explicit pairs, for callers that cannot give the library any device memory of
+ * their own to work in and cannot allocate at this point either: code running inside a memory-pool or
+ * allocator callback, under a framework that has claimed the whole device, or in a process whose
+ * policy forbids cudaMalloc after start-up.  (The paper has no counterpart; this is a convenience of
+ * this library.)  It computes exactly what regtopk_aggregate computes, g = sum_n omega_n * ghat_n with
+ * the workers added in the order 0..N-1, but takes the pairs as arguments and keeps its scratch (one
+ * bitmask row per worker) in a fixed array that is part of the library image instead of a workspace.
+ *   idx, val  [N][k] pairs as regtopk_worker_step writes them: per worker distinct indices in
+ *             ascending order.  omega: HOST array of N weights, or NULL for 1/N each.
+ *   out_g     [d] binary32, fully overwritten.
+ * Limits: N <= REGTOPK_STATIC_MAX_WORKERS and N * ceil(d/32 rounded up to 4) <= REGTOPK_STATIC_SCRATCH_WORDS
+ * (8 MiB of scratch, which every GPU that loads the library holds until the process exits); larger
+ * problems return REGTOPK_ERR_TOO_LARGE and must use a context.  No cudaMalloc, cudaFree or other
+ * allocating call is made.  The first call on each device looks up the scratch array's device address
+ * (that device must be current) and should therefore come before any stream capture.  All calls on a
+ * device share the one array and clear the part they use first: two calls whose work overlaps on the
+ * GPU (different streams, or different threads) race; issue them on one stream or synchronise between
+ * them.  Work is enqueued on cuda_stream; the call does not synchronise.
+ * Errors: INVALID_ARG, TOO_LARGE, NO_DEVICE, CUDA. */
+#define REGTOPK_STATIC_SCRATCH_WORDS (1u << 21)
+#define REGTOPK_STATIC_MAX_WORKERS 64
+int regtopk_aggregate_pairs_static(int64_t d, int32_t N, int64_t k, const int32_t* idx, const float* val,
+                                   const float* omega, float* out_g, void* cuda_stream);
 
 /* Frees the host-side context.  Synchronises the stream first.  The workspace is the caller's. */
 int regtopk_destroy(regtopk_ctx* ctx);

@@ -4,4 +4,4 @@
 in the CUDA library (csrc/regtopk.cu).  `synth` holds the seeded synthetic input generators; it
 contains none of the method's arithmetic.
 """
-from .binding import RegTopK, build, load_library, library_path  # noqa: F401
+from .binding import RegTopK, aggregate_pairs_static, build, load_library, library_path  # noqa: F401

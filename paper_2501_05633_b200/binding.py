@@ -26,7 +26,7 @@ EXPORTS = [
     "regtopk_workspace_bytes", "regtopk_create", "regtopk_worker_step", "regtopk_aggregate",
     "regtopk_global_gradient", "regtopk_state_reset", "regtopk_round_host", "regtopk_status",
     "regtopk_get_stats", "regtopk_profile_enable", "regtopk_profile_read", "regtopk_debug_residual",
-    "regtopk_destroy", "regtopk_strerror",
+    "regtopk_destroy", "regtopk_strerror", "regtopk_aggregate_pairs_static",
 ]
 
 
@@ -98,6 +98,8 @@ def load_library():
     L.regtopk_debug_residual.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i64)]
     L.regtopk_destroy.restype = ctypes.c_int
     L.regtopk_destroy.argtypes = [vp]
+    L.regtopk_aggregate_pairs_static.restype = ctypes.c_int
+    L.regtopk_aggregate_pairs_static.argtypes = [i64, i32, i64, vp, vp, ctypes.POINTER(ctypes.c_float), vp, vp]
     L.regtopk_strerror.restype = ctypes.c_char_p
     L.regtopk_strerror.argtypes = [ctypes.c_int]
     _lib = L
@@ -126,6 +128,33 @@ def _make_params(mu, omega, grad_dtype, flags):
     p.grad_dtype = grad_dtype
     p.flags = flags
     return p, keep
+
+
+STATIC_SCRATCH_WORDS = 1 << 21
+STATIC_MAX_WORKERS = 64
+
+
+def aggregate_pairs_static(idx: torch.Tensor, val: torch.Tensor, d: int, omega=None,
+                           out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """g = sum_n omega_n * ghat_n from explicit [N, k] pairs, using the library's built-in scratch
+    instead of a context's workspace.  For callers that must not allocate device memory around the call:
+    pass `out` (a [d] float32 device tensor made earlier) and nothing here allocates on the device.
+    Calls on one GPU share the scratch; keep them on one stream or synchronise between them."""
+    if not (idx.is_cuda and val.is_cuda and idx.dtype == torch.int32 and val.dtype == torch.float32):
+        raise TypeError("idx int32 and val float32 device tensors [N, k]")
+    idx, val = idx.contiguous(), val.contiguous()
+    N, k = idx.shape
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=idx.device)
+    om = None
+    if omega is not None:
+        om = (ctypes.c_float * N)(*[float(x) for x in omega])
+    s = stream if stream is not None else torch.cuda.current_stream(idx.device)
+    with torch.cuda.device(idx.device):
+        _check(load_library().regtopk_aggregate_pairs_static(d, N, k, idx.data_ptr(), val.data_ptr(), om,
+                                                             out.data_ptr(), s.cuda_stream),
+               "regtopk_aggregate_pairs_static")
+    return out
 
 
 def workspace_bytes(d, N, k, mu=4.0, omega=None, grad_dtype=GRAD_F32, flags=0) -> int:

@@ -1116,6 +1116,65 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Aggregation from explicit pairs with built-in scratch (regtopk_aggregate_pairs_static).
+// The scratch is a file-scope device array: it costs 8 MiB on every GPU that loads this library,
+// and it is shared by all calls on that GPU.  Host code never uses the symbol as a pointer; it asks
+// the runtime for the array's device address once per device.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) u32 g_static_scratch[REGTOPK_STATIC_SCRATCH_WORDS];
+
+struct StaticAggArgs {
+  float* g;
+  int N;
+  int64_t k;
+  const int32_t* idx;
+  const float* val;
+  u32* mask;  // [N][W], inside the static scratch, cleared by the caller of the kernels
+  int64_t W;
+  float omega[REGTOPK_STATIC_MAX_WORKERS];
+};
+
+__global__ void __launch_bounds__(256) k_static_mark(StaticAggArgs p) {
+  const int64_t total = p.k * p.N;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (int64_t)gridDim.x * blockDim.x) {
+    const int n = (int)(t / p.k);
+    const u32 j = (u32)p.idx[t];
+    atomicOr(&p.mask[(size_t)n * p.W + (j >> 5)], 1u << (j & 31));
+  }
+}
+
+// Same ownership rule as k_aggregate (the highest-numbered worker that sent j writes g[j], adding the
+// lower workers' terms in order); a lower worker's value is found by binary search in its ascending
+// index row instead of through the prefix directory a context keeps.
+__global__ void __launch_bounds__(256) k_static_aggregate(StaticAggArgs p) {
+  const int64_t total = p.k * p.N;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (int64_t)gridDim.x * blockDim.x) {
+    const int n = (int)(t / p.k);
+    const int32_t j = p.idx[t];
+    const size_t wi = (size_t)((u32)j >> 5);
+    const u32 bm = 1u << (j & 31);
+    bool owned = true;
+    for (int m = n + 1; m < p.N && owned; ++m) owned = !(p.mask[(size_t)m * p.W + wi] & bm);
+    if (!owned) continue;
+    float sum = 0.0f;
+    for (int m = 0; m < n; ++m) {
+      if (!(p.mask[(size_t)m * p.W + wi] & bm)) continue;
+      const int32_t* row = p.idx + (size_t)m * p.k;
+      int64_t lo = 0, hi = p.k;
+      while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (row[mid] < j) lo = mid + 1; else hi = mid;
+      }
+      sum = __fadd_rn(sum, __fmul_rn(p.omega[m], p.val[(size_t)m * p.k + lo]));
+    }
+    sum = __fadd_rn(sum, __fmul_rn(p.omega[n], p.val[t]));
+    p.g[j] = sum;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -1292,6 +1351,7 @@ const char* regtopk_strerror(int code) {
     case REGTOPK_ERR_CUDA: return "CUDA runtime error";
     case REGTOPK_ERR_INTERNAL: return "device reported an inconsistent selection";
     case REGTOPK_ERR_NO_DEVICE: return "no usable sm_100 device";
+    case REGTOPK_ERR_TOO_LARGE: return "problem exceeds the built-in static capacity (use a context with a workspace)";
     default: return "unknown error code";
   }
 }
@@ -1556,6 +1616,46 @@ int regtopk_debug_residual(regtopk_ctx* c, const float** dev_ptr, int64_t* ld) {
   if (!c || !dev_ptr || !ld) return REGTOPK_ERR_INVALID_ARG;
   *dev_ptr = at<float>(c, c->L.off_eps);
   *ld = c->L.ld;
+  return REGTOPK_OK;
+}
+
+int regtopk_aggregate_pairs_static(int64_t d, int32_t N, int64_t k, const int32_t* idx, const float* val,
+                                   const float* omega, float* out_g, void* cuda_stream) {
+  if (d < 1 || d > 2147483646LL || N < 1 || k < 1 || k > d || !idx || !val || !out_g)
+    return REGTOPK_ERR_INVALID_ARG;
+  if (N > REGTOPK_STATIC_MAX_WORKERS) return REGTOPK_ERR_TOO_LARGE;
+  const int64_t W = ((d + 31) / 32 + 3) / 4 * 4;
+  if ((int64_t)N * W > (int64_t)REGTOPK_STATIC_SCRATCH_WORDS) return REGTOPK_ERR_TOO_LARGE;
+  // Device address of the scratch array, looked up once per device with that device current.
+  static u32* scratch_of_device[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return REGTOPK_ERR_NO_DEVICE;
+  if (!scratch_of_device[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return REGTOPK_ERR_NO_DEVICE;
+    }
+    scratch_of_device[dev] = static_cast<u32*>(ptr);
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  StaticAggArgs a;
+  a.g = out_g; a.N = N; a.k = k; a.idx = idx; a.val = val; a.mask = scratch_of_device[dev]; a.W = W;
+  for (int n = 0; n < REGTOPK_STATIC_MAX_WORKERS; ++n) {
+    a.omega[n] = n < N ? (omega ? omega[n] : 1.0f / (float)N) : 0.0f;
+    if (n < N && !isfinite(a.omega[n])) return REGTOPK_ERR_INVALID_ARG;
+  }
+  // the array keeps the previous call's bits: clear the rows this call uses, and the whole output
+  if (cudaMemsetAsync(a.mask, 0, (size_t)N * W * sizeof(u32), stream) != cudaSuccess ||
+      cudaMemsetAsync(out_g, 0, (size_t)d * sizeof(float), stream) != cudaSuccess)
+    return REGTOPK_ERR_CUDA;
+  const int64_t total = k * (int64_t)N;
+  int64_t blocks = (total + 255) / 256;
+  if (blocks > 148 * 32) blocks = 148 * 32;
+  k_static_mark<<<(unsigned)blocks, 256, 0, stream>>>(a);
+  if (cudaGetLastError() != cudaSuccess) return REGTOPK_ERR_CUDA;
+  k_static_aggregate<<<(unsigned)blocks, 256, 0, stream>>>(a);
+  if (cudaGetLastError() != cudaSuccess) return REGTOPK_ERR_CUDA;
   return REGTOPK_OK;
 }
 
