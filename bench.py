@@ -22,6 +22,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_stream launch from the ncu capture summarised in
+# profiles/k_stream_resnet18_fp32_full.md; valid for that workload and the kernel as captured.
+NCU_STREAM_TRAFFIC = {"resnet18": 1021.7e6}
+
 METRIC = "RegTop-k step throughput (G coords/s, all N workers) and achieved HBM GB/s vs peak"
 UNIT = "G coords/s"
 
@@ -301,7 +305,8 @@ def main():
                     "h2d_bytes_per_step": w.N * stream.ld * bpe, "d2h_bytes_per_step": 2 * w.N * k * 4 + w.d * 4},
             "gpu_launches": launches,
             "roofline": {"bound": "hbm", "kernel": "k_stream", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                         "traffic": NCU_STREAM_TRAFFIC.get(w.name) if w.grad_dtype == "f32" else None,
                          "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": kern_avg_ms},
         }
         if world == 1 and not args.no_cpu_baseline:
