@@ -77,8 +77,8 @@ int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const reg
 /* One sparsification round of all N workers: Algorithm 2 steps 6-12 (Algorithm 1 steps 2-7 in round 0
  * or when mu == 0).
  *   grads    [N][grad_ld] gradients g_n^t in the context's grad_dtype, row n at grads + n*grad_ld
- *            elements; read-only.  grad_ld >= d.  Rows that are 16-byte aligned (fp32: grad_ld % 4 == 0
- *            and an aligned base; bf16: 8-byte, grad_ld % 4 == 0) take the vectorised path; any other
+ *            elements; read-only.  grad_ld >= d.  Rows that are 16-byte aligned (an aligned base and
+ *            grad_ld % 4 == 0 for fp32, grad_ld % 8 == 0 for bf16) take the vectorised path; any other
  *            layout is accepted and read element by element.
  *   out_idx  [N][k] int32: worker n's mask support in ascending order.
  *   out_val  [N][k] binary32: the accumulator a_n^t at those indices (not the score).
