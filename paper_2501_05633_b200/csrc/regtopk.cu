@@ -75,6 +75,15 @@ struct GlobalCtl {
   u64 dense_workers;
 };
 
+// Programmatic dependent launch: every kernel of the round is launched with the stream-serialization
+// attribute, lets its successor be scheduled at once (so that the successor's blocks take over SMs as
+// this kernel's blocks retire instead of after a full drain and launch), and itself waits here, before
+// its first memory access, until its predecessor has completed and its writes are visible.
+__device__ __forceinline__ void grid_dependency_begin() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ u64 make_composite(u32 key, u32 idx) {
   return (static_cast<u64>(key) << 32) | static_cast<u64>(kFull - idx);
 }
@@ -235,6 +244,7 @@ __device__ __forceinline__ void flush_hist(const u32* s_hist, u32* g_hist, int n
 template <bool BF16>
 __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
   extern __shared__ u32 s_hist[];  // kSampleBins bins, one pad word after every 16 (bank-conflict-free per-thread runs)
+  grid_dependency_begin();
   __shared__ u32 s_scan[33];
   __shared__ u32 s_res[3];
   cg::cluster_group cl = cg::this_cluster();
@@ -500,6 +510,7 @@ template <bool BF16, bool VEC>
 __global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC>::kBlocksPerSm) k_stream(StreamArgs p) {
   typedef StreamShape<BF16, VEC> S;
   __shared__ u64 s_list[kStreamThreads / 32][kWarpList];
+  grid_dependency_begin();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   u64* list = s_list[warp];
   u32 wcount = 0;  // warp-uniform
@@ -574,7 +585,8 @@ __global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC>::kBlock
         a.y = __fadd_rn(e[u][v].y, g[u][v].y);
         a.z = __fadd_rn(e[u][v].z, g[u][v].z);
         a.w = __fadd_rn(e[u][v].w, g[u][v].w);
-        *reinterpret_cast<float4*>(eps_row + j) = a;  // padding receives 0 + 0
+        __stcs(reinterpret_cast<float4*>(eps_row + j), a);  // padding receives 0 + 0; streaming store: the
+                                                            // accumulators should not push the small lists out of L2
         const u32 k0 = __float_as_uint(a.x) & 0x7FFFFFFFu, k1 = __float_as_uint(a.y) & 0x7FFFFFFFu;
         const u32 k2 = __float_as_uint(a.z) & 0x7FFFFFFFu, k3 = __float_as_uint(a.w) & 0x7FFFFFFFu;
         const bool h0 = k0 >= cutoff && (full || j + 0 < p.d);
@@ -767,6 +779,7 @@ __device__ __forceinline__ u32 popc4(const uint4& v) {
 
 __global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
   __shared__ __align__(16) PostShared sh;
+  grid_dependency_begin();
   cg::cluster_group cl = cg::this_cluster();
   const u32 CS = cl.num_blocks(), rk = cl.block_rank();
   const int n = blockIdx.x / CS;
@@ -852,19 +865,25 @@ __global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
 
   if (!dense) {
     // ---- classify: above the bin -> winner; inside it -> refinement list ----
-    // (each thread re-reads exactly the list slots it wrote or filtered before the barrier)
-    for (int part = 0; part < 2; ++part) {
-      const u64* items = part == 0 ? A : O;
-      const u32 count = part == 0 ? ncand : novr;
-      const u32 iters = (count + stride_t - 1) / stride_t;
+    // (candidates and overrides as one item list, eight loads per thread in flight)
+    {
+      const u32 total_items = ncand + novr;
+      const u32 iters = (total_items + 8 * stride_t - 1) / (8 * stride_t);
       for (u32 it = 0; it < iters; ++it) {
-        const u32 i = it * stride_t + first_t;
-        const u64 c = i < count ? items[i] : 0ull;
-        const u32 bin = c ? select_bin((u32)(c >> 32), cutoff, bshift) : 0u;
-        if (c && bin > b1) set_winner(mask, composite_idx(c));
-        const bool inbin = c && bin == b1;
-        const u32 pos = warp_reserve_global(inbin, &ctl->bcount);
-        if (inbin) B[pos] = c;
+        u64 c[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const u32 t = (it * 8 + q) * stride_t + first_t;
+          c[q] = t < ncand ? __ldcg(A + t) : (t < total_items ? __ldcg(O + (t - ncand)) : 0ull);
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const u32 bin = c[q] ? select_bin((u32)(c[q] >> 32), cutoff, bshift) : 0u;
+          if (c[q] && bin > b1) set_winner(mask, composite_idx(c[q]));
+          const bool inbin = c[q] && bin == b1;
+          const u32 pos = warp_reserve_global(inbin, &ctl->bcount);
+          if (inbin) B[pos] = c[q];
+        }
       }
     }
     cl.sync();  // (2) refinement list complete
@@ -964,26 +983,17 @@ __global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
   {
     const int64_t wu0 = (int64_t)gw * seg_units < U ? (int64_t)gw * seg_units : U;
     const int64_t wu1 = wu0 + seg_units < U ? wu0 + seg_units : U;
-    uint4 nx[2], ny[2];
-#pragma unroll
-    for (int it = 0; it < 2; ++it) {
-      const int64_t u = wu0 + it * 32 + lane;
-      nx[it] = u < wu1 ? __ldcg(quads + 2 * u) : make_uint4(0, 0, 0, 0);
-      ny[it] = u < wu1 ? __ldcg(quads + 2 * u + 1) : make_uint4(0, 0, 0, 0);
-    }
     u32 running = 0;
-    for (int64_t ub = wu0; ub < wu1; ub += 64) {
-      uint4 x[2], y[2];
+    for (int64_t ub = wu0; ub < wu1; ub += 128) {  // four rows of 32 units per step
+      uint4 x[4], y[4];
 #pragma unroll
-      for (int it = 0; it < 2; ++it) {
-        x[it] = nx[it];
-        y[it] = ny[it];
-        const int64_t u = ub + 64 + it * 32 + lane;  // next step's units, in flight during this step
-        nx[it] = u < wu1 ? __ldcg(quads + 2 * u) : make_uint4(0, 0, 0, 0);
-        ny[it] = u < wu1 ? __ldcg(quads + 2 * u + 1) : make_uint4(0, 0, 0, 0);
+      for (int it = 0; it < 4; ++it) {
+        const int64_t u = ub + it * 32 + lane;
+        x[it] = u < wu1 ? __ldcg(quads + 2 * u) : make_uint4(0, 0, 0, 0);
+        y[it] = u < wu1 ? __ldcg(quads + 2 * u + 1) : make_uint4(0, 0, 0, 0);
       }
 #pragma unroll
-      for (int it = 0; it < 2; ++it) {
+      for (int it = 0; it < 4; ++it) {
         const u32 cx = popc4(x[it]), c = cx + popc4(y[it]);
         u32 inc = c;
 #pragma unroll
@@ -1015,12 +1025,12 @@ __global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
       return;
     }
   }
-  for (int part = 0; part < 2; ++part) {
-    // normal path: candidates, then overrides; dense path: its k winners, nothing else.  Items
-    // below the threshold bin cannot have won and are skipped without touching memory.
-    const u64* items = part == 0 ? A : O;
-    const u32 count = part == 0 ? (took_dense ? k : ncand) : (took_dense ? 0u : novr);
-    for (u32 i0 = first_t; i0 < count; i0 += 4 * stride_t) {
+  {
+    // normal path: candidates and overrides as one item list; dense path: its k winners, nothing
+    // else.  Items below the threshold bin cannot have won and are skipped without touching memory.
+    const u32 nA = took_dense ? k : ncand;
+    const u32 total_items = nA + (took_dense ? 0u : novr);
+    for (u32 t0 = first_t; t0 < total_items; t0 += 4 * stride_t) {
       u64 c[4];
       uint4 qw[4];
       u32 qp[4];
@@ -1028,8 +1038,8 @@ __global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
       bool live[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const u32 i = i0 + q * stride_t;
-        c[q] = i < count ? __ldcg(items + i) : 0ull;
+        const u32 t = t0 + q * stride_t;
+        c[q] = t < nA ? __ldcg(A + t) : (t < total_items ? __ldcg(O + (t - nA)) : 0ull);
       }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
@@ -1091,6 +1101,7 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
   const int64_t npairs = p.k * p.N;
   const int64_t total = p.has_prev ? 2 * npairs : npairs;
   const int64_t Q = p.W >> 2;
+  grid_dependency_begin();
   for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
        t += (int64_t)gridDim.x * blockDim.x) {
     if (t >= npairs) {  // a pair of the previous round
@@ -1332,6 +1343,30 @@ int after_launch(regtopk_ctx* c) {
 
 size_t sample_smem() { return (size_t)kSamplePadded * sizeof(u32); }
 
+// Launch configuration: `blocks` blocks of `threads`, optionally in clusters, always with programmatic
+// stream serialization (see grid_dependency_begin).  attr must have room for two attributes.
+void launch_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, unsigned blocks, int cluster,
+                   int threads, size_t smem, cudaStream_t s) {
+  memset(cfg, 0, sizeof *cfg);
+  cfg->gridDim = dim3(blocks, 1, 1);
+  cfg->blockDim = dim3((unsigned)threads, 1, 1);
+  cfg->dynamicSmemBytes = smem;
+  cfg->stream = s;
+  int na = 0;
+  attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[na].val.programmaticStreamSerializationAllowed = 1;
+  ++na;
+  if (cluster > 1) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = (unsigned)cluster;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg->attrs = attr;
+  cfg->numAttrs = na;
+}
+
 template <bool BF16, bool VEC>
 void launch_stream(regtopk_ctx* c, const StreamArgs& a, int variant) {
   if (c->stream_blocks[variant] == 0) {
@@ -1344,22 +1379,15 @@ void launch_stream(regtopk_ctx* c, const StreamArgs& a, int variant) {
   const int64_t chunks = ((a.d + chunk - 1) / chunk) * a.N;
   int64_t blocks = (chunks + (kStreamThreads / 32) - 1) / (kStreamThreads / 32);
   if (blocks > c->stream_blocks[variant]) blocks = c->stream_blocks[variant];
-  k_stream<BF16, VEC><<<(unsigned)blocks, kStreamThreads, 0, c->stream>>>(a);
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[2];
+  launch_config(&cfg, attr, (unsigned)blocks, 1, kStreamThreads, 0, c->stream);
+  cudaLaunchKernelEx(&cfg, k_stream<BF16, VEC>, a);
 }
 
 void post_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int N, int cluster, int threads,
                  cudaStream_t s) {
-  memset(cfg, 0, sizeof *cfg);
-  cfg->gridDim = dim3((unsigned)(N * cluster), 1, 1);
-  cfg->blockDim = dim3((unsigned)threads, 1, 1);
-  cfg->dynamicSmemBytes = 0;
-  cfg->stream = s;
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)cluster;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg->attrs = attr;
-  cfg->numAttrs = 1;
+  launch_config(cfg, attr, (unsigned)(N * cluster), cluster, threads, 0, s);
 }
 
 // Blocks per worker for k_post: the largest power of two up to 16 (sizes above 8 need the
@@ -1371,7 +1399,7 @@ int choose_cluster(int N) {
   int schedulable = 1;
   for (int cs = kMaxCluster; cs > 1; cs >>= 1) {
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     post_config(&cfg, attr, N, cs, kBlockPost, nullptr);
     int nclusters = 0;
     if (cudaOccupancyMaxActiveClusters(&nclusters, k_post, &cfg) != cudaSuccess) {
@@ -1490,7 +1518,7 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   sa.force_dense = (c->flags & REGTOPK_FLAG_FORCE_DENSE_SELECT) ? 1 : 0;
   {
     cudaLaunchConfig_t scfg;
-    cudaLaunchAttribute sattr[1];
+    cudaLaunchAttribute sattr[2];
     int extra = use_marks ? (c->num_sms - c->N * kSampleCluster) / kSampleCluster : 0;  // override clusters
     if (use_marks && extra < 1) extra = 1;
     post_config(&scfg, sattr, c->N + extra, kSampleCluster, kBlockSel, c->stream);
@@ -1528,7 +1556,7 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   pa.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); pa.cur_val = at<float>(c, L.off_val[c->cur]);
   pa.use_marks = use_marks; pa.has_stale = c->round >= 2;
   cudaLaunchConfig_t cfg;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   post_config(&cfg, attr, c->N, c->cluster, kBlockPost, c->stream);
   cudaError_t le = cudaLaunchKernelEx(&cfg, k_post, pa);
   c->launches++;
@@ -1555,7 +1583,12 @@ int regtopk_aggregate(regtopk_ctx* c, float* out_g) {
   const int64_t threads = (a.has_prev ? 2 : 1) * c->k * (int64_t)c->N;
   int64_t blocks = (threads + 255) / 256;
   if (blocks > (int64_t)c->num_sms * 32) blocks = (int64_t)c->num_sms * 32;
-  k_aggregate<<<(unsigned)blocks, 256, 0, c->stream>>>(a);
+  {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    launch_config(&cfg, attr, (unsigned)blocks, 1, 256, 0, c->stream);
+    cudaLaunchKernelEx(&cfg, k_aggregate, a);
+  }
   int rc = after_launch(c);
   if (rc) return rc;
   if (out_g)
