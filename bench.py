@@ -33,7 +33,7 @@ UNIT = "G coords/s"
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet18", choices=["resnet18", "resnet50", "gpt2", "flat1p3b"])
@@ -170,7 +170,7 @@ def cpu_baseline(w, k, seed):
     from paper_2501_05633_b200 import synth
     from oracle.oracle import OracleRegTopK
     from oracle.oracle import grads_view as to_oracle_view
-    nw = min(w.N, 4)  # bounded: a full sort of d entries per worker costs about a second per 10M
+    nw = min(w.N, 8)  # bounded: a full sort of d entries per worker costs about a second per 10M
     wsamp = synth.workload(w.name)
     wsamp.N = nw
     stream = synth.GradientStream(wsamp, device="cuda", seed=seed)

@@ -293,3 +293,53 @@ def test_full_size_workloads(name, ki, rounds):
     s = synth.GradientStream(w, device="cuda", seed=0, pad_to=32)
     run_parity((s.next() for _ in range(rounds)), w.d, w.N, w.k_values()[ki], w.mu, select_mode=1, threads=8,
                expect_dense=False)
+
+
+# ---- full benchmark sizes too large to sort on the host: certified instead of compared --------------------------
+def _certified_round(lib, ora_api, w, k, grads, eps_before, prev, g_prev, omega):
+    """One round of the library, checked against the oracle without a sort: the oracle's accumulator and
+    scores are computed per worker (O(d)), the library's mask is certified as the selector's answer
+    (no record outside it ranks before its last-ranked record), and everything else is element-wise."""
+    idx, val = lib.worker_step(grads)
+    lib.status()
+    idx_h, val_h = idx.cpu().numpy(), val.cpu().numpy()
+    eps_after = lib.residual()
+    for n in range(w.N):
+        g_n = grads[n, : w.d].cpu()
+        g_view = g_n.view(torch.int16).numpy().view(np.uint16) if g_n.dtype == torch.bfloat16 else g_n.numpy()
+        pi, pv = (None, None) if prev is None else (prev[0][n], prev[1][n])
+        a, s = ora_api.scores(g_view, eps_before[n], pi, pv, g_prev, w.mu, float(omega[n]))
+        assert ora_api.mask_certificate(s, idx_h[n]) == k, f"worker {n}: not the k largest scores"
+        assert np.array_equal(val_h[n].view(np.uint32), a[idx_h[n]].view(np.uint32)), f"worker {n}: sent values"
+        a[idx_h[n]] = 0.0
+        assert np.array_equal(eps_after[n].cpu().numpy().view(np.uint32), a.view(np.uint32)), f"worker {n}: residual"
+        del a, s
+    agg = lib.aggregate().cpu().numpy()
+    want = ora_api.aggregate(w.d, omega, idx_h, val_h)
+    assert np.array_equal(agg.view(np.uint32), want.view(np.uint32)), "aggregate"
+    lib.status()
+    return (idx_h, val_h), agg
+
+
+@pytest.mark.parametrize("name,ki,rounds", [("gpt2", 0, 2), ("flat1p3b", 1, 2)])
+def test_full_size_certified(name, ki, rounds):
+    import psutil
+    from oracle.oracle import default as oracle_default
+    w = synth.workload(name)
+    need_host = 5 * w.N * w.d * 4  # residual copies, one worker's gradient, accumulator and scores
+    if psutil.virtual_memory().available < need_host:
+        pytest.skip("not enough host memory for the element-wise checks")
+    k = w.k_values()[ki]
+    tdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+    s = synth.GradientStream(w, device="cuda", seed=0, pad_to=32)
+    lib = RegTopK(w.d, w.N, k, mu=w.mu, grad_dtype=tdt)
+    omega = np.full(w.N, np.float32(1.0) / np.float32(w.N), np.float32)
+    eps_before = np.zeros((w.N, w.d), np.float32)
+    prev, g_prev = None, None
+    for t in range(rounds):
+        grads = s.next()
+        prev, g_prev = _certified_round(lib, oracle_default(), w, k, grads, eps_before, prev, g_prev, omega)
+        if t + 1 < rounds:
+            eps_before = lib.residual().cpu().numpy()
+        del grads
+    assert lib.stats()["dense_select_workers"] == 0
