@@ -481,17 +481,19 @@ __device__ __forceinline__ void stream_flush(u64* list, u32& wcount, WorkerCtl* 
   __syncwarp();
 }
 
-// Elements a lane handles per step and steps a warp keeps in flight.  What bounds this kernel is the
-// number of bytes in flight per SM (loaded HBM latency is about 2 us): fp32 keeps eight steps of four
-// elements per lane in flight (256 B per thread, two blocks per SM); the bf16 variant, whose gradient
-// loads are half as wide, takes eight elements per lane and step (16-byte gradient loads) and four steps.
-// Measured on a B200: fp32 4 -> 8 steps: 5.96 -> 6.17 TB/s on 89 M coordinates; bf16 with 8-byte gradient
-// loads: 3.8-4.9 TB/s, with 16-byte loads: 5.2 TB/s.
+// Elements a lane handles per step, steps a warp keeps in flight, and resident blocks per SM.  What
+// bounds this kernel is the number of bytes in flight per SM (loaded HBM latency is about 2 us) against
+// the registers that costs.  Shapes chosen by measurement on a B200:
+//   fp32: four elements per lane and step, eight steps (256 B per thread), two blocks per SM:
+//         6.17 TB/s on 89 M coordinates (four steps and three blocks: 5.96-6.09; four blocks: 5.80);
+//   bf16: eight elements per lane and step (one 16-byte gradient load), two steps (96 B per thread),
+//         three blocks per SM: 6.11 TB/s on 996 M coordinates (four steps, two blocks: 4.98-5.27;
+//         8-byte gradient loads: 3.8).
 #ifndef REGTOPK_STREAM_STEPS_F32
 #define REGTOPK_STREAM_STEPS_F32 8
 #endif
 #ifndef REGTOPK_STREAM_STEPS_BF16
-#define REGTOPK_STREAM_STEPS_BF16 4
+#define REGTOPK_STREAM_STEPS_BF16 2
 #endif
 #ifndef REGTOPK_STREAM_EPL_BF16
 #define REGTOPK_STREAM_EPL_BF16 8
@@ -503,7 +505,13 @@ struct StreamShape {
   static constexpr int kStep = 32 * kEpl;                   // elements per warp and step
   static constexpr int kSteps = (BF16 && VEC) ? REGTOPK_STREAM_STEPS_BF16 : (VEC ? REGTOPK_STREAM_STEPS_F32 : 4);
   static constexpr int kChunk = kStep * kSteps;             // elements per warp iteration (divides 1024)
-  static constexpr int kBlocksPerSm = kSteps * kEpl > 16 ? 2 : 3;
+#ifndef REGTOPK_STREAM_BLOCKS_F32
+#define REGTOPK_STREAM_BLOCKS_F32 2
+#endif
+#ifndef REGTOPK_STREAM_BLOCKS_BF16
+#define REGTOPK_STREAM_BLOCKS_BF16 3
+#endif
+  static constexpr int kBlocksPerSm = (BF16 && VEC) ? REGTOPK_STREAM_BLOCKS_BF16 : (VEC ? REGTOPK_STREAM_BLOCKS_F32 : 2);
 };
 
 template <bool BF16, bool VEC>
