@@ -231,6 +231,7 @@ struct SampleArgs {
   const float* omega;
   float mu;
   u32* ovr_key;             // [N][k] out: score bits
+  int share_override;       // the sampling blocks take a share of the override work too
 };
 
 // Add a block's histogram to the cluster's in global memory (non-empty bins only).
@@ -238,6 +239,49 @@ __device__ __forceinline__ void flush_hist(const u32* s_hist, u32* g_hist, int n
   for (int i = threadIdx.x; i < nbins; i += blockDim.x) {
     const u32 v = s_hist[i];
     if (v) atomicAdd(&g_hist[i], v);
+  }
+}
+
+// Regularised scores of the previous support (Eq. (Delta_def), Algorithm 2 steps 8-9) for the items
+// first, first + nthreads, ... of the N*k previous pairs; four items per thread in flight.
+template <bool BF16>
+__device__ __forceinline__ void override_scores(const SampleArgs& p, int64_t first, int64_t nthreads) {
+  const int64_t total = p.k * p.N;
+  for (int64_t t0 = first; t0 < total; t0 += 4 * nthreads) {
+    int32_t j[4];
+    float ap[4], G[4], gr[4];
+    int wn[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int64_t t = t0 + q * nthreads;
+      const bool in = t < total;
+      j[q] = in ? p.prev_idx[t] : 0;
+      ap[q] = in ? p.prev_val[t] : 0.0f;
+      wn[q] = in ? (int)(t / p.k) : 0;
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const bool in = t0 + q * nthreads < total;
+      G[q] = in ? p.g_prev[j[q]] : 0.0f;
+      gr[q] = in ? load_grad<BF16>(static_cast<const char*>(p.grads) + (size_t)wn[q] * p.grad_ld * (BF16 ? 2 : 4), j[q]) : 0.0f;
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int64_t t = t0 + q * nthreads;
+      if (t < total) {
+        const float w = p.omega[wn[q]];
+        const float a = __fadd_rn(0.0f, gr[q]);
+        const float num = __fsub_rn(G[q], __fmul_rn(w, ap[q]));
+        const float den = __fmul_rn(w, a);
+        float m = 1.0f;
+        if (den != 0.0f) {
+          const float delta = __fdiv_rn(num, den);
+          const float r = fabsf(__fadd_rn(1.0f, delta));
+          m = tanh_fixed(__fdiv_rn(r, p.mu));
+        }
+        p.ovr_key[t] = __float_as_uint(__fmul_rn(fabsf(a), m));
+      }
+    }
   }
 }
 
@@ -253,47 +297,16 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
   const int tid = threadIdx.x;
   if (n >= p.N) {  // an override cluster: no barriers on this path
     if (!p.use_marks) return;
-    const int64_t total = p.k * p.N;
-    const int64_t nthreads = (int64_t)(gridDim.x - p.N * kSampleCluster) * blockDim.x;
-    const int64_t first = (int64_t)(blockIdx.x - p.N * kSampleCluster) * blockDim.x + tid;
-    for (int64_t t0 = first; t0 < total; t0 += 4 * nthreads) {
-      int32_t j[4];
-      float ap[4], G[4], gr[4];
-      int wn[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int64_t t = t0 + q * nthreads;
-        const bool in = t < total;
-        j[q] = in ? p.prev_idx[t] : 0;
-        ap[q] = in ? p.prev_val[t] : 0.0f;
-        wn[q] = in ? (int)(t / p.k) : 0;
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const bool in = t0 + q * nthreads < total;
-        G[q] = in ? p.g_prev[j[q]] : 0.0f;
-        gr[q] = in ? load_grad<BF16>(static_cast<const char*>(p.grads) + (size_t)wn[q] * p.grad_ld * (BF16 ? 2 : 4), j[q]) : 0.0f;
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int64_t t = t0 + q * nthreads;
-        if (t < total) {
-          const float w = p.omega[wn[q]];
-          const float a = __fadd_rn(0.0f, gr[q]);
-          const float num = __fsub_rn(G[q], __fmul_rn(w, ap[q]));
-          const float den = __fmul_rn(w, a);
-          float m = 1.0f;
-          if (den != 0.0f) {
-            const float delta = __fdiv_rn(num, den);
-            const float r = fabsf(__fadd_rn(1.0f, delta));
-            m = tanh_fixed(__fdiv_rn(r, p.mu));
-          }
-          p.ovr_key[t] = __float_as_uint(__fmul_rn(fabsf(a), m));
-        }
-      }
-    }
+    if (p.share_override)
+      override_scores<BF16>(p, (int64_t)blockIdx.x * blockDim.x + tid, (int64_t)gridDim.x * blockDim.x);
+    else
+      override_scores<BF16>(p, (int64_t)(blockIdx.x - p.N * kSampleCluster) * blockDim.x + tid,
+                            (int64_t)(gridDim.x - p.N * kSampleCluster) * blockDim.x);
     return;
   }
+  // with many overrides the sampling blocks take their share of them first (the sampling itself is short)
+  if (p.use_marks && p.share_override)
+    override_scores<BF16>(p, (int64_t)blockIdx.x * blockDim.x + tid, (int64_t)gridDim.x * blockDim.x);
   WorkerCtl* ctl = p.ctl + n;
   u32* shist = p.shist + (size_t)n * kSampleBins;
 
@@ -1523,12 +1536,14 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   sa.N = c->N; sa.use_marks = use_marks; sa.g_prev = at<float>(c, L.off_g);
   sa.prev_idx = at<int32_t>(c, L.off_idx[prev]); sa.prev_val = at<float>(c, L.off_val[prev]);
   sa.omega = at<float>(c, L.off_omega); sa.mu = c->mu; sa.ovr_key = at<u32>(c, L.off_ovr_key);
+  sa.share_override = 0;
   sa.force_dense = (c->flags & REGTOPK_FLAG_FORCE_DENSE_SELECT) ? 1 : 0;
   {
     cudaLaunchConfig_t scfg;
     cudaLaunchAttribute sattr[2];
     int extra = use_marks ? (c->num_sms - c->N * kSampleCluster) / kSampleCluster : 0;  // override clusters
     if (use_marks && extra < 1) extra = 1;
+    sa.share_override = use_marks && c->k * (int64_t)c->N > (int64_t)4 * extra * kSampleCluster * kBlockSel;
     post_config(&scfg, sattr, c->N + extra, kSampleCluster, kBlockSel, c->stream);
     scfg.dynamicSmemBytes = sample_smem();
     cudaError_t se = bf16 ? cudaLaunchKernelEx(&scfg, k_sample_cutoff<true>, sa)
