@@ -1,19 +1,22 @@
 // RegTop-k sparsification step for N workers batched on one B200 (sm_100a): kernels and C ABI.
 //
-// One round (regtopk_worker_step + regtopk_aggregate) is four kernels on one stream:
+// One round (regtopk_worker_step + regtopk_aggregate) is four kernels on one stream, chained with
+// programmatic dependent launch:
 //
-//   k_sample_cutoff   one block per worker: reads a strided sample of a = eps + g and derives, from
-//                     the sample's order statistics, a candidate cutoff key (a guess that only has to
-//                     be low enough) and the bin width the select will use
+//   k_sample_cutoff   a cluster of 8 blocks per worker reads a strided sample of a = eps + g and
+//                     derives, from the sample's order statistics, a candidate cutoff key (a guess that
+//                     only has to be low enough) and the bin width the select will use.  Further
+//                     clusters of the same launch compute the regularised scores on the previous mask's
+//                     support (Eq. (Delta_def), Algorithm 2 steps 8-9) meanwhile.
 //   k_stream          the one Theta(N*d) pass: a = eps + g written in place over eps; every entry
-//                     whose key bits(|a|) reaches the cutoff is appended to the worker's candidate list
-//   k_post            one thread-block cluster per worker (distributed shared memory for the
-//                     histogram merge): regularised scores on the previous mask's support
-//                     (Eq. (Delta_def), Algorithm 2 steps 8-9), exact selection of the k largest
-//                     (score, lowest index) among candidates and overrides, winners set in a bitmask,
-//                     ordered walk of the bitmask emitting ascending (index, a[index]) pairs and
-//                     zeroing the residual there.  If the cutoff guess was too high or the list
-//                     overflowed, the same cluster runs an exact radix select over the whole row.
+//                     whose key bits(|a|) reaches the cutoff and that is not on the previous support is
+//                     appended to the worker's candidate list
+//   k_post            one thread-block cluster per worker: exact selection of the k largest (score,
+//                     lowest index) among candidates and overrides, winners set in a bitmask; per-quad
+//                     prefix counts of the bitmask give every winner its rank, and each winner writes
+//                     its (index, a[index]) pair there and zeroes its residual.  If the cutoff guess was
+//                     too high or the list overflowed, the same cluster runs an exact radix select over
+//                     the whole row.
 //   k_aggregate       server sum in worker order, one thread per sent pair, ranks looked up through
 //                     the prefix counts written during emission
 //

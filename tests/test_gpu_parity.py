@@ -27,7 +27,8 @@ def gauss_rounds(N, d, T, seed, ld=None, scale=None, dtype=torch.float32, quant=
 # ---- tiny and ragged sizes, every k regime -----------------------------------------------------------
 @pytest.mark.parametrize("d,N,k", [(1, 1, 1), (2, 2, 1), (7, 3, 7), (33, 2, 5), (511, 2, 17), (512, 1, 512),
                                    (513, 3, 1), (4096, 8, 41), (65536, 2, 100), (65537, 2, 655),
-                                   (200003, 4, 2000), (200003, 2, 200003), (1_000_003, 2, 1000)])
+                                   (200003, 4, 2000), (200003, 2, 200003), (1_000_003, 2, 1000),
+                                   (5000, 20, 50), (3001, 33, 7), (70_000, 150, 70)])
 @pytest.mark.parametrize("mu", [4.0, 0.0])
 def test_sizes(d, N, k, mu):
     run_parity(gauss_rounds(N, d, 4, seed=d + N), d, N, k, mu)
