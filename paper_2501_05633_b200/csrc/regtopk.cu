@@ -51,7 +51,10 @@ typedef uint32_t u32;
 constexpr int kSampleSectors = 8192;       // 32-byte sectors sampled per worker
 constexpr int kSampleMax = kSampleSectors * 8;
 constexpr int kBlockSel = 1024;            // threads per block of k_sample_cutoff
-constexpr int kBlockPost = 1024;           // threads per block of k_post
+#ifndef REGTOPK_POST_THREADS
+#define REGTOPK_POST_THREADS 1024
+#endif
+constexpr int kBlockPost = REGTOPK_POST_THREADS;  // threads per block of k_post
 constexpr int kStreamThreads = 256;
 constexpr int kWarpList = 256;             // per-warp staging list of k_stream (entries)
 constexpr int kBins = 4096;                // histogram bins of the select
@@ -801,7 +804,7 @@ __device__ __forceinline__ u32 popc4(const uint4& v) {
   return (u32)(__popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w));
 }
 
-__global__ void __launch_bounds__(kBlockPost, 1) k_post(PostArgs p) {
+__global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs p) {
   __shared__ __align__(16) PostShared sh;
   grid_dependency_begin();
   cg::cluster_group cl = cg::this_cluster();

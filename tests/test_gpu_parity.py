@@ -116,6 +116,26 @@ def test_denormals_and_huge_values():
     run_parity(rounds, d, N, 600, 4.0)
 
 
+def test_non_finite_inputs_do_not_break_the_context():
+    """Gradients must be finite; if they are not, the result is unspecified but nothing faults, exactly k
+    distinct ascending indices still come out, and after a reset the context is exact again."""
+    d, N, k = 50_000, 2, 500
+    lib = RegTopK(d, N, k)
+    g = torch.randn(N, d)
+    g[0, 10] = float("nan")
+    g[0, 11] = float("inf")
+    g[1, 12] = float("-inf")
+    for _ in range(3):
+        idx, _ = lib.worker_step(g.cuda())
+        lib.aggregate()
+        torch.cuda.synchronize()
+        ih = idx.cpu().numpy()
+        assert np.all(np.diff(ih, axis=1) > 0) and ih.min() >= 0 and ih.max() < d
+    assert lib.stats()["device_error_bits"] == 0
+    lib.close()
+    run_parity(gauss_rounds(N, d, 3, seed=77), d, N, k, 4.0)
+
+
 # ---- the dense exact path --------------------------------------------------------------------------------
 @pytest.mark.parametrize("mu", [4.0, 0.0])
 def test_forced_dense_select(mu):

@@ -1,5 +1,5 @@
 """Each plausible mistake, planted in a copy of the oracle's source on the CPU, must fail at least one
-pin.  This is what shows the pins are strong enough to trust the oracle as the judge of the CUDA path."""
+pin.  This is what shows the pins are strong enough to trust the oracle as the yardstick for the CUDA path."""
 import os
 import subprocess
 
