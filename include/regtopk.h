@@ -94,12 +94,31 @@ int regtopk_worker_step(regtopk_ctx* ctx, const void* grads, int64_t grad_ld, in
  * Errors: SEQUENCE (no worker_step since the last aggregate), CUDA. */
 int regtopk_aggregate(regtopk_ctx* ctx, float* out_g);
 
+/* regtopk_aggregate fused with the model update of distributed SGD (Section 1: theta^{t+1} = theta^t -
+ * eta^t g^t): after g^t is formed, theta[j] <- theta[j] - (eta * g^t[j]) (product rounded first) for every j
+ * some worker sent; all other entries would change by eta * 0 and are left alone, which is the same
+ * result bit for bit.  theta [d] binary32 (device), eta finite.  theta == NULL is regtopk_aggregate.
+ * Errors as regtopk_aggregate, plus INVALID_ARG for a non-finite eta. */
+int regtopk_aggregate_update(regtopk_ctx* ctx, float* theta, float eta, float* out_g);
+
 /* Device pointer to the library's own copy of the latest aggregate g^t ([d] binary32, inside the
  * workspace, valid until the next regtopk_aggregate is enqueued).  *dev_ptr is written on the host. */
 int regtopk_global_gradient(regtopk_ctx* ctx, const float** dev_ptr);
 
 /* Back to Algorithm 2's initial state: eps = 0, no previous mask, g = 0, round 0. */
 int regtopk_state_reset(regtopk_ctx* ctx);
+
+/* Checkpointing.  What Algorithm 2 carries from round to round (the residuals eps_n, the previous masks and the
+ * accumulator values on them, the previous aggregate g^{t-1}, the round counter) can be copied out of the workspace
+ * into a caller buffer of regtopk_state_bytes(ctx) bytes (device memory) and later copied into a context created
+ * with the same d, N, k, mu and grad_dtype; the rounds that follow are then bit-identical to the ones the exporting
+ * context would have run.  Export only between rounds (after regtopk_aggregate): otherwise SEQUENCE.
+ * regtopk_state_export enqueues the copies on the context's stream; regtopk_state_import synchronises the stream
+ * (it reads the blob's header) and returns INVALID_ARG if the blob does not belong to an identical problem,
+ * WORKSPACE_TOO_SMALL if `bytes` is short. */
+size_t regtopk_state_bytes(regtopk_ctx* ctx);
+int regtopk_state_export(regtopk_ctx* ctx, void* dst, size_t bytes);
+int regtopk_state_import(regtopk_ctx* ctx, const void* src, size_t bytes);
 
 /* One whole round from HOST buffers: copies h_grads ([N][grad_ld], pinned memory recommended) to the
  * device staging area, runs regtopk_worker_step and regtopk_aggregate, copies the pairs (and g if

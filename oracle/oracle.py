@@ -46,6 +46,8 @@ def _bind(path):
                                              _vp, _vp, _c_f32, _c_f32, _vp, _vp, ctypes.c_int]
     L.regtopk_oracle_aggregate.restype = None
     L.regtopk_oracle_aggregate.argtypes = [_c_i64, _c_i32, _c_i64, _vp, _vp, _vp, _vp]
+    L.regtopk_oracle_model_update.restype = None
+    L.regtopk_oracle_model_update.argtypes = [_c_i64, _vp, _c_f32, _vp]
     L.regtopk_oracle_mask_certificate.restype = _c_i64
     L.regtopk_oracle_mask_certificate.argtypes = [_c_i64, _c_i64, _vp, _vp]
     return L
@@ -123,6 +125,13 @@ class OracleAPI:
         g = np.empty(d, np.float32)
         self.L.regtopk_oracle_aggregate(d, N, k, _p(omega), _p(idx), _p(val), _p(g))
         return g
+
+    def model_update(self, theta, eta, g):
+        """theta <- theta - eta * g in place (theta float32, contiguous)."""
+        assert theta.dtype == np.float32 and theta.flags.c_contiguous
+        g = np.ascontiguousarray(g, dtype=np.float32)
+        self.L.regtopk_oracle_model_update(theta.shape[0], _p(theta), eta, _p(g))
+        return theta
 
     def mask_certificate(self, score, sel_idx):
         score = np.ascontiguousarray(score, dtype=np.float32)

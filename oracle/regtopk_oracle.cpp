@@ -14,6 +14,7 @@
 //   sparsified gradient = mask * a  (raw accumulator values)        Algorithm 2 steps 10-11
 //   residual          eps' = a - ghat                               Algorithm 1 step 7, Algorithm 2 step 12
 //   server            g = sum_n w_n * ghat_n                        Section 2.2 (aggregation equation)
+//   model update      theta' = theta - eta * g                      Section 1 (after Eq. (1))
 //
 // Readings taken where the paper is silent (each listed in the design notes):
 //   * ties in the magnitude sort: the lower index wins;
@@ -194,6 +195,15 @@ void regtopk_oracle_aggregate(int64_t d, int32_t N, int64_t k, const float* omeg
       int64_t j = idx[n * k + i];
       g_out[j] = g_out[j] + t;
     }
+  }
+}
+
+// Model update of distributed SGD, theta^{t+1} = theta^t - eta * g^t (Section 1, after Eq. (1)), in place;
+// the product is rounded before the subtraction.
+void regtopk_oracle_model_update(int64_t d, float* theta, float eta, const float* g) {
+  for (int64_t j = 0; j < d; ++j) {
+    float step = eta * g[j];
+    theta[j] = theta[j] - step;
   }
 }
 

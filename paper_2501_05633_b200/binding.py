@@ -26,7 +26,8 @@ EXPORTS = [
     "regtopk_workspace_bytes", "regtopk_create", "regtopk_worker_step", "regtopk_aggregate",
     "regtopk_global_gradient", "regtopk_state_reset", "regtopk_round_host", "regtopk_status",
     "regtopk_get_stats", "regtopk_profile_enable", "regtopk_profile_read", "regtopk_debug_residual",
-    "regtopk_destroy", "regtopk_strerror", "regtopk_aggregate_pairs_static",
+    "regtopk_destroy", "regtopk_strerror", "regtopk_aggregate_pairs_static", "regtopk_aggregate_update", "regtopk_state_bytes",
+    "regtopk_state_export", "regtopk_state_import",
 ]
 
 
@@ -80,6 +81,14 @@ def load_library():
     L.regtopk_worker_step.argtypes = [vp, vp, i64, vp, vp]
     L.regtopk_aggregate.restype = ctypes.c_int
     L.regtopk_aggregate.argtypes = [vp, vp]
+    L.regtopk_aggregate_update.restype = ctypes.c_int
+    L.regtopk_aggregate_update.argtypes = [vp, vp, ctypes.c_float, vp]
+    L.regtopk_state_bytes.restype = ctypes.c_size_t
+    L.regtopk_state_bytes.argtypes = [vp]
+    L.regtopk_state_export.restype = ctypes.c_int
+    L.regtopk_state_export.argtypes = [vp, vp, ctypes.c_size_t]
+    L.regtopk_state_import.restype = ctypes.c_int
+    L.regtopk_state_import.argtypes = [vp, vp, ctypes.c_size_t]
     L.regtopk_global_gradient.restype = ctypes.c_int
     L.regtopk_global_gradient.argtypes = [vp, ctypes.POINTER(vp)]
     L.regtopk_state_reset.restype = ctypes.c_int
@@ -232,6 +241,27 @@ class RegTopK:
         _check(self.L.regtopk_aggregate(self.ctx, out.data_ptr() if out is not None else None),
                "regtopk_aggregate")
         return out if out is not None else self.global_gradient()
+
+    def aggregate_update(self, theta: torch.Tensor, eta: float, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """aggregate() fused with theta <- theta - eta * g (theta: [d] float32 on the device, updated in place)."""
+        if not (theta.is_cuda and theta.dtype == torch.float32 and theta.is_contiguous() and theta.numel() == self.d):
+            raise TypeError("theta must be a contiguous [d] float32 device tensor")
+        _check(self.L.regtopk_aggregate_update(self.ctx, theta.data_ptr(), float(eta),
+                                               out.data_ptr() if out is not None else None),
+               "regtopk_aggregate_update")
+        return out if out is not None else self.global_gradient()
+
+    def state_export(self) -> torch.Tensor:
+        """The state carried between rounds as one uint8 device tensor (call between rounds)."""
+        n = int(self.L.regtopk_state_bytes(self.ctx))
+        blob = torch.empty(n, dtype=torch.uint8, device=self.device)
+        _check(self.L.regtopk_state_export(self.ctx, blob.data_ptr(), n), "regtopk_state_export")
+        return blob
+
+    def state_import(self, blob: torch.Tensor):
+        if not (blob.is_cuda and blob.dtype == torch.uint8 and blob.is_contiguous()):
+            raise TypeError("state blob must be a contiguous uint8 device tensor")
+        _check(self.L.regtopk_state_import(self.ctx, blob.data_ptr(), blob.numel()), "regtopk_state_import")
 
     def global_gradient(self) -> torch.Tensor:
         """View of the library's g^t inside the workspace (overwritten by the next aggregate)."""

@@ -1122,6 +1122,8 @@ struct AggArgs {
   int64_t W;
   const float* omega;
   int has_prev;
+  float* theta;  // optional model vector: theta[j] <- theta[j] - eta * g[j] where g[j] was written
+  float eta;
 };
 
 __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
@@ -1195,6 +1197,8 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
     }
     sum = __fadd_rn(sum, __fmul_rn(p.omega[n], p.cur_val[t]));
     p.g[j] = sum;
+    // theta - eta * 0 is theta, so updating only where the aggregate is non-trivial is the dense update
+    if (p.theta) p.theta[j] = __fsub_rn(p.theta[j], __fmul_rn(p.eta, sum));
   }
 }
 
@@ -1596,8 +1600,10 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   return REGTOPK_OK;
 }
 
-int regtopk_aggregate(regtopk_ctx* c, float* out_g) {
-  if (!c) return REGTOPK_ERR_INVALID_ARG;
+int regtopk_aggregate(regtopk_ctx* c, float* out_g) { return regtopk_aggregate_update(c, nullptr, 0.0f, out_g); }
+
+int regtopk_aggregate_update(regtopk_ctx* c, float* theta, float eta, float* out_g) {
+  if (!c || (theta && !isfinite(eta))) return REGTOPK_ERR_INVALID_ARG;
   if (!c->stepped) return REGTOPK_ERR_SEQUENCE;
   const Layout& L = c->L;
   AggArgs a;
@@ -1609,6 +1615,7 @@ int regtopk_aggregate(regtopk_ctx* c, float* out_g) {
   a.W = L.W;
   a.omega = at<float>(c, L.off_omega);
   a.has_prev = c->round >= 1;
+  a.theta = theta; a.eta = eta;
   const int64_t threads = (a.has_prev ? 2 : 1) * c->k * (int64_t)c->N;
   int64_t blocks = (threads + 255) / 256;
   if (blocks > (int64_t)c->num_sms * 32) blocks = (int64_t)c->num_sms * 32;
@@ -1632,6 +1639,67 @@ int regtopk_global_gradient(regtopk_ctx* c, const float** dev_ptr) {
   if (!c || !dev_ptr) return REGTOPK_ERR_INVALID_ARG;
   *dev_ptr = at<float>(c, c->L.off_g);
   return REGTOPK_OK;
+}
+
+namespace {
+struct StateHeader {
+  uint64_t magic;
+  int64_t d, k, ld, W, round;
+  int32_t N, cur, grad_dtype;
+  uint32_t mu_bits;
+};
+constexpr uint64_t kStateMagic = 0x52544B5354415445ull;  // "RTKSTATE"
+constexpr size_t kStateHeaderBytes = 256;
+size_t state_part1(const Layout& L) { return L.off_ctl; }                      // residuals, g, both masks
+size_t state_part2(const Layout& L) { return L.off_ovr_key - L.off_idx[0]; }   // both pair buffers
+}  // namespace
+
+size_t regtopk_state_bytes(regtopk_ctx* c) {
+  if (!c) return 0;
+  return kStateHeaderBytes + state_part1(c->L) + state_part2(c->L);
+}
+
+int regtopk_state_export(regtopk_ctx* c, void* dst, size_t bytes) {
+  if (!c || !dst) return REGTOPK_ERR_INVALID_ARG;
+  if (bytes < regtopk_state_bytes(c)) return REGTOPK_ERR_WORKSPACE_TOO_SMALL;
+  if (c->stepped) return REGTOPK_ERR_SEQUENCE;
+  char hdr[kStateHeaderBytes];
+  memset(hdr, 0, sizeof hdr);
+  StateHeader h;
+  h.magic = kStateMagic; h.d = c->d; h.k = c->k; h.ld = c->L.ld; h.W = c->L.W; h.round = c->round;
+  h.N = c->N; h.cur = c->cur; h.grad_dtype = c->grad_dtype;
+  memcpy(&h.mu_bits, &c->mu, 4);
+  memcpy(hdr, &h, sizeof h);
+  char* out = static_cast<char*>(dst);
+  // the header is pageable host memory: the runtime stages it before cudaMemcpyAsync returns
+  int rc = note_cuda(c, cudaMemcpyAsync(out, hdr, kStateHeaderBytes, cudaMemcpyHostToDevice, c->stream));
+  if (!rc) rc = note_cuda(c, cudaMemcpyAsync(out + kStateHeaderBytes, c->ws, state_part1(c->L),
+                                            cudaMemcpyDeviceToDevice, c->stream));
+  if (!rc) rc = note_cuda(c, cudaMemcpyAsync(out + kStateHeaderBytes + state_part1(c->L), c->ws + c->L.off_idx[0],
+                                            state_part2(c->L), cudaMemcpyDeviceToDevice, c->stream));
+  return rc;
+}
+
+int regtopk_state_import(regtopk_ctx* c, const void* src, size_t bytes) {
+  if (!c || !src) return REGTOPK_ERR_INVALID_ARG;
+  if (bytes < regtopk_state_bytes(c)) return REGTOPK_ERR_WORKSPACE_TOO_SMALL;
+  const char* in = static_cast<const char*>(src);
+  StateHeader h;
+  int rc = note_cuda(c, cudaMemcpyAsync(&h, in, sizeof h, cudaMemcpyDeviceToHost, c->stream));
+  if (!rc) rc = note_cuda(c, cudaStreamSynchronize(c->stream));
+  if (rc) return rc;
+  uint32_t mu_bits;
+  memcpy(&mu_bits, &c->mu, 4);
+  if (h.magic != kStateMagic || h.d != c->d || h.k != c->k || h.N != c->N || h.ld != c->L.ld || h.W != c->L.W ||
+      h.grad_dtype != c->grad_dtype || h.mu_bits != mu_bits || h.round < 0 || (h.cur != 0 && h.cur != 1))
+    return REGTOPK_ERR_INVALID_ARG;
+  rc = regtopk_state_reset(c);  // clears the control blocks and histograms as well
+  if (!rc) rc = note_cuda(c, cudaMemcpyAsync(c->ws, in + kStateHeaderBytes, state_part1(c->L),
+                                            cudaMemcpyDeviceToDevice, c->stream));
+  if (!rc) rc = note_cuda(c, cudaMemcpyAsync(c->ws + c->L.off_idx[0], in + kStateHeaderBytes + state_part1(c->L),
+                                            state_part2(c->L), cudaMemcpyDeviceToDevice, c->stream));
+  if (!rc) { c->round = h.round; c->cur = h.cur; c->stepped = 0; }
+  return rc;
 }
 
 int regtopk_round_host(regtopk_ctx* c, const void* h_grads, int64_t grad_ld, int32_t* h_idx,

@@ -278,6 +278,23 @@ def pin_aggregation(api):
     assert g[1] == np.float32(np.float32(np.float32(0) + t0) + t1)
 
 
+def pin_model_update(api):
+    """theta' = theta - eta*g with the product rounded first; entries with g = 0 keep their bits (also -0)."""
+    theta = np.array([1.0, -0.0, 0.5, 2.0, 1.0], np.float32)
+    g = np.array([2.0, 0.0, -1.0, 0.0, 3.3], np.float32)
+    out = api.model_update(theta.copy(), 0.5, g)
+    assert np.array_equal(out[:4], np.array([0.0, -0.0, 1.0, 2.0], np.float32)) and np.signbit(out[1])
+    # not a power of two: two roundings, in this order
+    out = api.model_update(theta.copy(), 0.1, g)
+    want = np.float32(np.float32(1.0) - np.float32(np.float32(0.1) * np.float32(3.3)))
+    assert out[4] == want
+    # exact cancellation that a fused multiply-subtract would miss: eta*g rounds to 1 exactly
+    e = np.float32(1.0) + np.float32(2.0 ** -23)
+    gg = np.array([np.float32(1.0) - np.float32(2.0 ** -24)], np.float32)
+    out = api.model_update(np.array([1.0], np.float32), float(e), gg)
+    assert out[0] == np.float32(np.float32(1.0) - np.float32(e * gg[0]))
+
+
 def pin_bf16_gradients(api):
     """bfloat16 gradients are widened exactly before the binary32 add."""
     bits = np.array([0x3F80, 0xBF00, 0x0000, 0x4049, 0x8000], np.uint16)  # 1, -0.5, 0, 3.140625, -0
@@ -320,5 +337,5 @@ def pin_mask_certificate(api):
 
 ALL_PINS = [pin_tanh, pin_bruteforce_selector, pin_dense_passthrough, pin_reduces_to_topk,
             pin_error_feedback_identity, pin_toy_example, pin_table1_iteration1, pin_distortion_cases,
-            pin_regularised_ranking, pin_aggregation, pin_bf16_gradients, pin_select_modes_agree,
+            pin_regularised_ranking, pin_aggregation, pin_model_update, pin_bf16_gradients, pin_select_modes_agree,
             pin_mask_certificate]

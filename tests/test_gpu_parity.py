@@ -216,6 +216,64 @@ def test_least_squares_trajectory():
     assert losses[50] < losses[0]
 
 
+def test_fused_model_update_trajectory():
+    """theta <- theta - eta*g fused into the aggregation (Section 1): the fp32 model vector stays bit-identical to
+    the oracle's over 40 rounds of the least-squares problem, and the loss falls."""
+    from oracle.oracle import OracleRegTopK, default as oracle_default
+    prob = synth.LeastSquares(N=4, rows=256, d=2048, seed=3)
+    k, eta = 40, 0.1
+    lib = RegTopK(prob.d, prob.N, k, mu=4.0)
+    ora = OracleRegTopK(prob.d, prob.N, k, 4.0)
+    th_dev = torch.zeros(prob.d, device="cuda")
+    th_ora = np.zeros(prob.d, np.float32)
+    first = prob.loss(th_ora.astype(np.float64))
+    for t in range(40):
+        g = prob.gradients(th_ora.astype(np.float64))
+        idx, val = lib.worker_step(torch.from_numpy(g).cuda())
+        oi, ov = ora.worker_step(g)
+        assert np.array_equal(idx.cpu().numpy(), oi)
+        agg = lib.aggregate_update(th_dev, eta)
+        oracle_default().model_update(th_ora, eta, ora.aggregate())
+        assert np.array_equal(agg.cpu().numpy().view(np.uint32), ora.g_prev.view(np.uint32))
+        assert np.array_equal(th_dev.cpu().numpy().view(np.uint32), th_ora.view(np.uint32)), f"round {t}"
+    lib.status()
+    assert prob.loss(th_ora.astype(np.float64)) < 0.9 * first
+
+
+def test_state_export_import_resumes_bit_identically():
+    d, N, k = 150_001, 3, 1500
+    rounds = [x.cuda() for x in gauss_rounds(N, d, 7, seed=91)]
+    a = RegTopK(d, N, k)
+    for g in rounds[:4]:
+        a.worker_step(g)
+        a.aggregate()
+    blob = a.state_export()
+    a.worker_step(rounds[4])
+    with pytest.raises(RegTopKError) as e:  # mid-round: refused
+        a.state_export()
+    assert e.value.code == -3
+    a.aggregate()
+    ref = []
+    for g in rounds[5:]:
+        idx, val = a.worker_step(g)
+        ref.append((idx.clone(), val.clone(), a.aggregate().clone(), a.residual().clone()))
+    b = RegTopK(d, N, k)
+    b.state_import(blob)
+    b.worker_step(rounds[4])
+    b.aggregate()
+    for g, want in zip(rounds[5:], ref):
+        idx, val = b.worker_step(g)
+        got = (idx, val, b.aggregate(), b.residual())
+        for x, y in zip(got, want):
+            assert torch.equal(x, y)
+    b.status()
+    other = RegTopK(d, N, k + 1)
+    with pytest.raises(RegTopKError):  # a blob of a different problem
+        other.state_import(blob)
+    with pytest.raises(RegTopKError):
+        b.state_import(blob[:1000].clone())
+
+
 # ---- API behaviour -------------------------------------------------------------------------------------------
 def test_state_reset_restarts_at_round_zero():
     run_parity(gauss_rounds(2, 20_000, 6, seed=40), 20_000, 2, 200, 4.0, reset_after=3)

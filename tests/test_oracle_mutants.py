@@ -33,6 +33,8 @@ MUTANTS = [
     ("aggregate_no_weight", "float t = omega[n] * val[n * k + i];", "float t = val[n * k + i];"),
     ("aggregate_overwrites", "g_out[j] = g_out[j] + t;", "g_out[j] = t;"),
     ("aggregate_reverse_order", "for (int32_t n = 0; n < N; ++n) {", "for (int32_t n = N - 1; n >= 0; --n) {"),
+    ("update_adds", "theta[j] = theta[j] - step;", "theta[j] = theta[j] + step;"),
+    ("update_ignores_eta", "float step = eta * g[j];", "float step = g[j];"),
     ("tanh_inverted", "return (1.0f - t) / (1.0f + t);", "return (1.0f + t) / (1.0f - t);"),
     ("tanh_exp_minus_x", "float y = (-2.0f * x) * log2e;", "float y = (-1.0f * x) * log2e;"),
     ("tanh_small_branch_linear", "return x + x * q;", "return x;"),
