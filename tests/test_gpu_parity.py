@@ -216,6 +216,36 @@ def test_least_squares_trajectory():
     assert losses[50] < losses[0]
 
 
+def test_toy_logistic_example_on_the_library():
+    """The paper's motivational example (Section 1.3: J = 2, two workers with x = [+-100, 1], eta = 0.9,
+    theta0 = [0, 1]) run on the library: Top-1 keeps sending the cancelling first coordinate and the loss does
+    not move for 90 rounds; RegTop-1 sees Delta = -1 exactly at t = 1, switches to the second coordinate and
+    the loss falls.  Same picks as the oracle every round."""
+    from oracle.oracle import OracleRegTopK
+    from tests.oracle_pins import _toy_gradients, _toy_loss
+    for mu in (0.0, 1.0):
+        lib = RegTopK(2, 2, 1, mu=mu)
+        ora = OracleRegTopK(2, 2, 1, mu)
+        theta = np.array([0.0, 1.0])
+        losses = [_toy_loss(theta)]
+        picks = []
+        for t in range(100):
+            g = _toy_gradients(theta)
+            idx, val = lib.worker_step(torch.from_numpy(g).cuda())
+            oi, ov = ora.worker_step(g)
+            assert np.array_equal(idx.cpu().numpy(), oi) and np.array_equal(val.cpu().numpy(), ov)
+            agg = lib.aggregate().cpu().numpy()
+            assert np.array_equal(agg.view(np.uint32), ora.aggregate().view(np.uint32))
+            theta = theta - 0.9 * agg.astype(np.float64)
+            picks.append(tuple(int(i) for i in idx.cpu().numpy()[:, 0]))
+            losses.append(_toy_loss(theta))
+        lib.status()
+        if mu == 0.0:
+            assert all(p == (0, 0) for p in picks[:90]) and all(l == losses[0] for l in losses[:91])
+        else:
+            assert picks[0] == (0, 0) and picks[1] == (1, 1) and losses[30] < 0.5 * losses[0]
+
+
 def test_fused_model_update_trajectory():
     """theta <- theta - eta*g fused into the aggregation (Section 1): the fp32 model vector stays bit-identical to
     the oracle's over 40 rounds of the least-squares problem, and the loss falls."""
