@@ -59,6 +59,9 @@ typedef struct {
   const float* omega;  /* host array of N aggregation weights (Eq. (1)), or NULL for 1/N each.             */
   int32_t grad_dtype;  /* REGTOPK_GRAD_F32 or REGTOPK_GRAD_BF16; accumulators and residuals are binary32.  */
   int32_t flags;       /* REGTOPK_FLAG_*                                                                   */
+  float y;             /* exponent of Remark 3: selection metric |a|^y * regulariser, 0 < y <= 1; 0 or 1 means
+                          Algorithm 2 as printed.  The mask is computed by ranking |a| * regulariser^(1/y), which
+                          orders the entries the same way.                                                   */
 } regtopk_params;
 
 /* Bytes of device workspace a context for (d, N, k) needs; 0 if the arguments are invalid.
@@ -111,7 +114,7 @@ int regtopk_state_reset(regtopk_ctx* ctx);
 /* Checkpointing.  What Algorithm 2 carries from round to round (the residuals eps_n, the previous masks and the
  * accumulator values on them, the previous aggregate g^{t-1}, the round counter) can be copied out of the workspace
  * into a caller buffer of regtopk_state_bytes(ctx) bytes (device memory) and later copied into a context created
- * with the same d, N, k, mu and grad_dtype; the rounds that follow are then bit-identical to the ones the exporting
+ * with the same d, N, k, mu, y and grad_dtype; the rounds that follow are then bit-identical to the ones the exporting
  * context would have run.  Export only between rounds (after regtopk_aggregate): otherwise SEQUENCE.
  * regtopk_state_export enqueues the copies on the context's stream; regtopk_state_import synchronises the stream
  * (it reads the blob's header) and returns INVALID_ARG if the blob does not belong to an identical problem,

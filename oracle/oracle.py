@@ -39,11 +39,13 @@ def _bind(path):
     L.regtopk_oracle_tanh.restype = _c_f32
     L.regtopk_oracle_tanh.argtypes = [_c_f32]
     L.regtopk_oracle_scores.restype = None
+    L.regtopk_oracle_pow.restype = _c_f32
+    L.regtopk_oracle_pow.argtypes = [_c_f32, _c_f32]
     L.regtopk_oracle_scores.argtypes = [_c_i64, _vp, ctypes.c_int, _vp, _c_i64, _vp, _vp, _vp,
-                                        _c_f32, _c_f32, _vp, _vp]
+                                        _c_f32, _c_f32, _c_f32, _vp, _vp]
     L.regtopk_oracle_worker_step.restype = ctypes.c_int
     L.regtopk_oracle_worker_step.argtypes = [_c_i64, _c_i64, _vp, ctypes.c_int, _vp, _c_i64, _vp,
-                                             _vp, _vp, _c_f32, _c_f32, _vp, _vp, ctypes.c_int]
+                                             _vp, _vp, _c_f32, _c_f32, _c_f32, _vp, _vp, ctypes.c_int]
     L.regtopk_oracle_aggregate.restype = None
     L.regtopk_oracle_aggregate.argtypes = [_c_i64, _c_i32, _c_i64, _vp, _vp, _vp, _vp]
     L.regtopk_oracle_model_update.restype = None
@@ -90,7 +92,15 @@ class OracleAPI:
             fo[i] = self.L.regtopk_oracle_tanh(_c_f32(float(fi[i])))
         return out
 
-    def scores(self, grad, eps, prev_idx, prev_val, g_prev, mu, omega_n):
+    def pow_spec(self, m, p) -> np.ndarray:
+        m = np.asarray(m, dtype=np.float32)
+        out = np.empty_like(m)
+        fi, fo = m.reshape(-1), out.reshape(-1)
+        for i in range(fi.size):
+            fo[i] = self.L.regtopk_oracle_pow(_c_f32(float(fi[i])), _c_f32(float(p)))
+        return out
+
+    def scores(self, grad, eps, prev_idx, prev_val, g_prev, mu, omega_n, y=1.0):
         """(a, score) of one worker; prev_idx=None means no previous round."""
         grad, code = _grad_view(grad)
         d = grad.shape[0]
@@ -99,10 +109,10 @@ class OracleAPI:
         s = np.empty(d, np.float32)
         n_prev, pi, pv, gp = _prev_views(prev_idx, prev_val, g_prev)
         self.L.regtopk_oracle_scores(d, _p(grad), code, _p(eps), n_prev, _p(pi), _p(pv), _p(gp),
-                                     mu, omega_n, _p(a), _p(s))
+                                     mu, omega_n, y, _p(a), _p(s))
         return a, s
 
-    def worker_step(self, grad, eps, k, prev_idx, prev_val, g_prev, mu, omega_n, select_mode=0):
+    def worker_step(self, grad, eps, k, prev_idx, prev_val, g_prev, mu, omega_n, select_mode=0, y=1.0):
         """One worker, one round. eps (float32, contiguous) is updated in place. Returns (idx, val)."""
         grad, code = _grad_view(grad)
         d = grad.shape[0]
@@ -111,10 +121,10 @@ class OracleAPI:
         out_val = np.empty(k, np.float32)
         n_prev, pi, pv, gp = _prev_views(prev_idx, prev_val, g_prev)
         rc = self.L.regtopk_oracle_worker_step(d, k, _p(grad), code, _p(eps), n_prev, _p(pi),
-                                               _p(pv), _p(gp), mu, omega_n, _p(out_idx),
+                                               _p(pv), _p(gp), mu, omega_n, y, _p(out_idx),
                                                _p(out_val), select_mode)
         if rc != 0:
-            raise ValueError("oracle rejected the sizes (need 1 <= k <= d < 2^31)")
+            raise ValueError("oracle rejected the arguments (need 1 <= k <= d < 2^31, 0 < y <= 1)")
         return out_idx, out_val
 
     def aggregate(self, d, omega, idx, val):
@@ -166,8 +176,9 @@ class OracleRegTopK:
     independent workers over host threads; each worker's computation is unchanged.
     """
 
-    def __init__(self, d, N, k, mu, omega=None, select_mode=0, threads=1, api=None):
+    def __init__(self, d, N, k, mu, omega=None, select_mode=0, threads=1, api=None, y=1.0):
         self.api = api or default()
+        self.y = float(y)
         self.d, self.N, self.k, self.mu = int(d), int(N), int(k), float(mu)
         self.omega = (np.full(N, np.float32(1.0) / np.float32(N), np.float32) if omega is None
                       else np.asarray(omega, np.float32).copy())
@@ -188,7 +199,7 @@ class OracleRegTopK:
         pi = None if self.prev_idx is None else self.prev_idx[n]
         pv = None if self.prev_val is None else self.prev_val[n]
         return self.api.worker_step(grads[n], self.eps[n], self.k, pi, pv, self.g_prev, self.mu,
-                           float(self.omega[n]), self.select_mode)
+                           float(self.omega[n]), self.select_mode, self.y)
 
     def worker_step(self, grads):
         assert grads.shape == (self.N, self.d)

@@ -11,6 +11,7 @@
 //   posterior distortion  Delta = (g_prev - w*a_prev) / (w*a)       Eq. (Delta_def), Algorithm 2 step 8
 //   regularised score |a| * tanh(|1 + Delta| / mu) on the previous support, |a| elsewhere (C = 1)
 //                                                                   Section 4, Algorithm 2 step 9
+//   exponent variant  metric |a|^y * regulariser, y <= 1            Remark 3 (appendix)
 //   sparsified gradient = mask * a  (raw accumulator values)        Algorithm 2 steps 10-11
 //   residual          eps' = a - ghat                               Algorithm 1 step 7, Algorithm 2 step 12
 //   server            g = sum_n w_n * ghat_n                        Section 2.2 (aggregation equation)
@@ -112,6 +113,56 @@ float regtopk_oracle_tanh(float x) {
   return (1.0f - t) / (1.0f + t);
 }
 
+// m^p for 0 <= m <= 1 and p >= 1 as a fixed sequence of binary32 operations (used for the exponent
+// variant of Remark 3): 0 -> 0, 1 -> 1, otherwise 2^(p * log2 m) with
+//   log2 m = e + log2 f, m = 2^e f, f in (sqrt(1/2), sqrt 2]; ln f = 2 s (1 + s2/3 + s2^2/5 + s2^3/7 + s2^4/9),
+//   s = (f - 1)/(f + 1), s2 = s*s (Horner); log2 f = ln f * log2(e);
+//   2^z as in regtopk_oracle_tanh (n = nearest integer, degree-7 polynomial of 2^(z - n), exact scaling);
+//   z < -125 -> 0.
+float regtopk_oracle_pow(float m, float p) {
+  if (m == 0.0f) return 0.0f;
+  if (m >= 1.0f) return 1.0f;
+  int e0 = 0;
+  if (m < 0x1p-126f) {  // subnormal: scale into the normal range (exact)
+    m = m * 0x1p+24f;
+    e0 = -24;
+  }
+  uint32_t b;
+  std::memcpy(&b, &m, sizeof b);
+  int e = static_cast<int>((b >> 23) & 0xffu) - 127 + e0;
+  uint32_t fb = (b & 0x7fffffu) | 0x3f800000u;
+  float f;
+  std::memcpy(&f, &fb, sizeof f);
+  if (f > 0x1.6a09e6p+0f) {  // sqrt(2)
+    f = f * 0.5f;
+    e += 1;
+  }
+  float s = (f - 1.0f) / (f + 1.0f);
+  float s2 = s * s;
+  float q = 0x1.c71c72p-4f;            // 1/9
+  q = 0x1.24924ap-3f + s2 * q;         // 1/7
+  q = 0x1.99999ap-3f + s2 * q;         // 1/5
+  q = 0x1.555556p-2f + s2 * q;         // 1/3
+  q = 1.0f + s2 * q;
+  float lnf = (2.0f * s) * q;
+  float log2f = lnf * 0x1.715476p+0f;  // log2(e)
+  float L = static_cast<float>(e) + log2f;
+  float z = p * L;
+  if (!(z >= -125.0f)) return 0.0f;
+  const float e1 = 0x1.62e430p-1f, e2 = 0x1.ebfbe0p-3f, e3 = 0x1.c6b08ep-5f, e4 = 0x1.3b2ab6p-7f;
+  const float e5 = 0x1.5d87fep-10f, e6 = 0x1.430912p-13f, e7 = 0x1.ffcbfcp-17f;
+  float n = std::nearbyintf(z);
+  float fr = z - n;
+  float P = e6 + fr * e7;
+  P = e5 + fr * P;
+  P = e4 + fr * P;
+  P = e3 + fr * P;
+  P = e2 + fr * P;
+  P = e1 + fr * P;
+  P = 1.0f + fr * P;
+  return std::ldexp(P, static_cast<int>(n));  // n in [-125, 0]: exact scaling
+}
+
 // Accumulator and selection score of one worker (Algorithm 2 steps 7-9).
 //   grad        d gradient entries, binary32 (grad_dtype 0) or bfloat16 bit patterns (grad_dtype 1)
 //   eps         d residual entries carried from the previous round
@@ -121,10 +172,13 @@ float regtopk_oracle_tanh(float x) {
 //   g_prev      d entries: the previous aggregated sparse gradient g^{t-1}
 //   mu          regulariser parameter; mu == 0 selects plain Top-k (no regularisation)
 //   omega_n     this worker's aggregation weight
+//   y           exponent of Remark 3 (selection metric |a|^y * regulariser), 0 < y <= 1; y = 1 is Algorithm 2.
+//               Ranking by |a|^y * m is ranking by |a| * m^(1/y); the score is computed in the second form,
+//               which leaves the score off the previous support equal to |a|
 //   a_out, score_out   d entries each
 void regtopk_oracle_scores(int64_t d, const void* grad, int grad_dtype, const float* eps,
                            int64_t n_prev, const int32_t* prev_idx, const float* prev_val,
-                           const float* g_prev, float mu, float omega_n, float* a_out,
+                           const float* g_prev, float mu, float omega_n, float y, float* a_out,
                            float* score_out) {
   for (int64_t j = 0; j < d; ++j) {
     float a = eps[j] + grad_at(grad, grad_dtype, j);
@@ -146,6 +200,7 @@ void regtopk_oracle_scores(int64_t d, const void* grad, int grad_dtype, const fl
         float x = r / mu;
         m = regtopk_oracle_tanh(x);
       }
+      if (y != 1.0f) m = regtopk_oracle_pow(m, 1.0f / y);
       score_out[j] = std::fabs(a) * m;
     }
   }
@@ -158,11 +213,11 @@ void regtopk_oracle_scores(int64_t d, const void* grad, int grad_dtype, const fl
 // mode 0 by the tests).  Returns 0, or -1 on invalid sizes.
 int regtopk_oracle_worker_step(int64_t d, int64_t k, const void* grad, int grad_dtype, float* eps,
                                int64_t n_prev, const int32_t* prev_idx, const float* prev_val,
-                               const float* g_prev, float mu, float omega_n, int32_t* out_idx,
+                               const float* g_prev, float mu, float omega_n, float y, int32_t* out_idx,
                                float* out_val, int select_mode) {
-  if (d < 1 || k < 1 || k > d || d > INT32_MAX) return -1;
+  if (d < 1 || k < 1 || k > d || d > INT32_MAX || !(y > 0.0f && y <= 1.0f)) return -1;
   std::vector<float> a(d), score(d);
-  regtopk_oracle_scores(d, grad, grad_dtype, eps, n_prev, prev_idx, prev_val, g_prev, mu, omega_n,
+  regtopk_oracle_scores(d, grad, grad_dtype, eps, n_prev, prev_idx, prev_val, g_prev, mu, omega_n, y,
                         a.data(), score.data());
   std::vector<Scored> rec(d);
   for (int64_t j = 0; j < d; ++j) rec[j] = Scored{score[j], static_cast<int32_t>(j)};

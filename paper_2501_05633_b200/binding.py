@@ -33,7 +33,7 @@ EXPORTS = [
 
 class Params(ctypes.Structure):
     _fields_ = [("mu", ctypes.c_float), ("omega", ctypes.POINTER(ctypes.c_float)),
-                ("grad_dtype", ctypes.c_int32), ("flags", ctypes.c_int32)]
+                ("grad_dtype", ctypes.c_int32), ("flags", ctypes.c_int32), ("y", ctypes.c_float)]
 
 
 class Stats(ctypes.Structure):
@@ -127,7 +127,7 @@ def _check(code: int, where: str):
         raise RegTopKError(code, where)
 
 
-def _make_params(mu, omega, grad_dtype, flags):
+def _make_params(mu, omega, grad_dtype, flags, y=1.0):
     p = Params()
     p.mu = float(mu)
     keep = None
@@ -136,6 +136,7 @@ def _make_params(mu, omega, grad_dtype, flags):
         p.omega = ctypes.cast(keep, ctypes.POINTER(ctypes.c_float))
     p.grad_dtype = grad_dtype
     p.flags = flags
+    p.y = float(y)
     return p, keep
 
 
@@ -166,8 +167,8 @@ def aggregate_pairs_static(idx: torch.Tensor, val: torch.Tensor, d: int, omega=N
     return out
 
 
-def workspace_bytes(d, N, k, mu=4.0, omega=None, grad_dtype=GRAD_F32, flags=0) -> int:
-    p, _keep = _make_params(mu, omega, grad_dtype, flags)
+def workspace_bytes(d, N, k, mu=4.0, omega=None, grad_dtype=GRAD_F32, flags=0, y=1.0) -> int:
+    p, _keep = _make_params(mu, omega, grad_dtype, flags, y)
     return int(load_library().regtopk_workspace_bytes(d, N, k, ctypes.byref(p)))
 
 
@@ -181,7 +182,7 @@ class RegTopK:
     """
 
     def __init__(self, d: int, N: int, k: int, mu: float = 4.0, omega=None, grad_dtype=torch.float32,
-                 flags: int = 0, device=None, stream: Optional[torch.cuda.Stream] = None):
+                 flags: int = 0, device=None, stream: Optional[torch.cuda.Stream] = None, y: float = 1.0):
         if not torch.cuda.is_available():
             raise RuntimeError("RegTopK needs a CUDA device; there is no CPU implementation")
         self.L = load_library()
@@ -192,7 +193,8 @@ class RegTopK:
         if grad_dtype not in (torch.float32, torch.bfloat16):
             raise TypeError("gradients are float32 or bfloat16")
         self.flags = int(flags)
-        p, keep = _make_params(mu, omega, self.dtype_code, self.flags)
+        self.y = float(y)
+        p, keep = _make_params(mu, omega, self.dtype_code, self.flags, self.y)
         nbytes = int(self.L.regtopk_workspace_bytes(self.d, self.N, self.k, ctypes.byref(p)))
         if nbytes == 0:
             raise RegTopKError(-1, "regtopk_workspace_bytes")

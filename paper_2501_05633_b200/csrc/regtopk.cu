@@ -191,6 +191,49 @@ __device__ __forceinline__ float tanh_fixed(float x) {
   return __fdiv_rn(__fsub_rn(1.0f, t), __fadd_rn(1.0f, t));
 }
 
+// m^p for 0 <= m <= 1, p >= 1 (exponent variant of Remark 3), as a fixed sequence of individually
+// rounded binary32 operations: 0 -> 0, 1 -> 1, else 2^(p * log2 m); log2 m = e + log2 f with m = 2^e f,
+// f in (sqrt(1/2), sqrt 2], ln f = 2 s (1 + s2/3 + s2^2/5 + s2^3/7 + s2^4/9), s = (f - 1)/(f + 1);
+// 2^z by the polynomial of tanh_fixed; z < -125 -> 0.
+__device__ __forceinline__ float pow_fixed(float m, float p) {
+  if (m == 0.0f) return 0.0f;
+  if (m >= 1.0f) return 1.0f;
+  int e0 = 0;
+  if (m < __uint_as_float(0x00800000u)) {  // subnormal: exact scaling into the normal range
+    m = __fmul_rn(m, 16777216.0f);
+    e0 = -24;
+  }
+  const u32 b = __float_as_uint(m);
+  int e = (int)((b >> 23) & 0xffu) - 127 + e0;
+  float f = __uint_as_float((b & 0x7fffffu) | 0x3f800000u);
+  if (f > __uint_as_float(0x3fb504f3u)) {  // sqrt(2)
+    f = __fmul_rn(f, 0.5f);
+    e += 1;
+  }
+  const float s = __fdiv_rn(__fsub_rn(f, 1.0f), __fadd_rn(f, 1.0f));
+  const float s2 = __fmul_rn(s, s);
+  float q = __uint_as_float(0x3de38e39u);                                    // 1/9
+  q = __fadd_rn(__uint_as_float(0x3e124925u), __fmul_rn(s2, q));             // 1/7
+  q = __fadd_rn(__uint_as_float(0x3e4ccccdu), __fmul_rn(s2, q));             // 1/5
+  q = __fadd_rn(__uint_as_float(0x3eaaaaabu), __fmul_rn(s2, q));             // 1/3
+  q = __fadd_rn(1.0f, __fmul_rn(s2, q));
+  const float lnf = __fmul_rn(__fmul_rn(2.0f, s), q);
+  const float log2f = __fmul_rn(lnf, __uint_as_float(0x3fb8aa3bu));
+  const float L = __fadd_rn((float)e, log2f);
+  const float z = __fmul_rn(p, L);
+  if (!(z >= -125.0f)) return 0.0f;
+  const float n = rintf(z);
+  const float fr = __fsub_rn(z, n);
+  float P = __fadd_rn(__uint_as_float(0x39218489u), __fmul_rn(fr, __uint_as_float(0x377fe5feu)));
+  P = __fadd_rn(__uint_as_float(0x3aaec3ffu), __fmul_rn(fr, P));
+  P = __fadd_rn(__uint_as_float(0x3c1d955bu), __fmul_rn(fr, P));
+  P = __fadd_rn(__uint_as_float(0x3d635847u), __fmul_rn(fr, P));
+  P = __fadd_rn(__uint_as_float(0x3e75fdf0u), __fmul_rn(fr, P));
+  P = __fadd_rn(__uint_as_float(0x3f317218u), __fmul_rn(fr, P));
+  P = __fadd_rn(1.0f, __fmul_rn(fr, P));
+  return __fmul_rn(P, __uint_as_float((u32)((int)n + 127) << 23));  // n in [-125, 0]: exact scaling
+}
+
 template <bool BF16>
 __device__ __forceinline__ float load_grad(const void* row, int64_t j) {
   if (BF16) {
@@ -236,6 +279,7 @@ struct SampleArgs {
   const float* prev_val;    // [N][k]
   const float* omega;
   float mu;
+  float inv_y;              // 1/y of the exponent variant (1: Algorithm 2 as printed)
   u32* ovr_key;             // [N][k] out: score bits
   int share_override;       // the sampling blocks take a share of the override work too
 };
@@ -285,6 +329,7 @@ __device__ __forceinline__ void override_scores(const SampleArgs& p, int64_t fir
           const float r = fabsf(__fadd_rn(1.0f, delta));
           m = tanh_fixed(__fdiv_rn(r, p.mu));
         }
+        if (p.inv_y != 1.0f) m = pow_fixed(m, p.inv_y);  // Remark 3: rank by |a|^y m, i.e. by |a| m^(1/y)
         p.ovr_key[t] = __float_as_uint(__fmul_rn(fabsf(a), m));
       }
     }
@@ -1277,6 +1322,7 @@ bool valid_problem(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
   if (!pr) return false;
   if (d < 1 || d > 2147483646LL || N < 1 || N > 65535 || k < 1 || k > d) return false;
   if (!(pr->mu >= 0.0f) || !isfinite(pr->mu)) return false;
+  if (!(pr->y >= 0.0f && pr->y <= 1.0f)) return false;  // 0 means "not set": y = 1
   if (pr->grad_dtype != REGTOPK_GRAD_F32 && pr->grad_dtype != REGTOPK_GRAD_BF16) return false;
   if (pr->omega)
     for (int n = 0; n < N; ++n)
@@ -1337,7 +1383,7 @@ constexpr int kMaxProfile = 4096;
 struct regtopk_ctx {
   int64_t d, k;
   int32_t N;
-  float mu;
+  float mu, inv_y;
   int32_t grad_dtype, flags;
   Layout L;
   char* ws;
@@ -1500,6 +1546,7 @@ int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const reg
   if (!c) return REGTOPK_ERR_INVALID_ARG;
   c->d = d; c->k = k; c->N = N;
   c->mu = params->mu;
+  c->inv_y = (params->y == 0.0f || params->y == 1.0f) ? 1.0f : 1.0f / params->y;
   c->grad_dtype = params->grad_dtype;
   c->flags = params->flags;
   c->L = L;
@@ -1545,7 +1592,7 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   sa.ghist = at<u32>(c, L.off_ghist);
   sa.N = c->N; sa.use_marks = use_marks; sa.g_prev = at<float>(c, L.off_g);
   sa.prev_idx = at<int32_t>(c, L.off_idx[prev]); sa.prev_val = at<float>(c, L.off_val[prev]);
-  sa.omega = at<float>(c, L.off_omega); sa.mu = c->mu; sa.ovr_key = at<u32>(c, L.off_ovr_key);
+  sa.omega = at<float>(c, L.off_omega); sa.mu = c->mu; sa.inv_y = c->inv_y; sa.ovr_key = at<u32>(c, L.off_ovr_key);
   sa.share_override = 0;
   sa.force_dense = (c->flags & REGTOPK_FLAG_FORCE_DENSE_SELECT) ? 1 : 0;
   {
@@ -1646,7 +1693,7 @@ struct StateHeader {
   uint64_t magic;
   int64_t d, k, ld, W, round;
   int32_t N, cur, grad_dtype;
-  uint32_t mu_bits;
+  uint32_t mu_bits, inv_y_bits;
 };
 constexpr uint64_t kStateMagic = 0x52544B5354415445ull;  // "RTKSTATE"
 constexpr size_t kStateHeaderBytes = 256;
@@ -1669,6 +1716,7 @@ int regtopk_state_export(regtopk_ctx* c, void* dst, size_t bytes) {
   h.magic = kStateMagic; h.d = c->d; h.k = c->k; h.ld = c->L.ld; h.W = c->L.W; h.round = c->round;
   h.N = c->N; h.cur = c->cur; h.grad_dtype = c->grad_dtype;
   memcpy(&h.mu_bits, &c->mu, 4);
+  memcpy(&h.inv_y_bits, &c->inv_y, 4);
   memcpy(hdr, &h, sizeof h);
   char* out = static_cast<char*>(dst);
   // the header is pageable host memory: the runtime stages it before cudaMemcpyAsync returns
@@ -1688,10 +1736,11 @@ int regtopk_state_import(regtopk_ctx* c, const void* src, size_t bytes) {
   int rc = note_cuda(c, cudaMemcpyAsync(&h, in, sizeof h, cudaMemcpyDeviceToHost, c->stream));
   if (!rc) rc = note_cuda(c, cudaStreamSynchronize(c->stream));
   if (rc) return rc;
-  uint32_t mu_bits;
+  uint32_t mu_bits, inv_y_bits;
   memcpy(&mu_bits, &c->mu, 4);
+  memcpy(&inv_y_bits, &c->inv_y, 4);
   if (h.magic != kStateMagic || h.d != c->d || h.k != c->k || h.N != c->N || h.ld != c->L.ld || h.W != c->L.W ||
-      h.grad_dtype != c->grad_dtype || h.mu_bits != mu_bits || h.round < 0 || (h.cur != 0 && h.cur != 1))
+      h.grad_dtype != c->grad_dtype || h.mu_bits != mu_bits || h.inv_y_bits != inv_y_bits || h.round < 0 || (h.cur != 0 && h.cur != 1))
     return REGTOPK_ERR_INVALID_ARG;
   rc = regtopk_state_reset(c);  // clears the control blocks and histograms as well
   if (!rc) rc = note_cuda(c, cudaMemcpyAsync(c->ws, in + kStateHeaderBytes, state_part1(c->L),

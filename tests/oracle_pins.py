@@ -278,6 +278,64 @@ def pin_aggregation(api):
     assert g[1] == np.float32(np.float32(np.float32(0) + t0) + t1)
 
 
+def pin_pow(api):
+    m = np.concatenate([np.linspace(1e-6, 1, 4001), np.logspace(-30, 0, 600)]).astype(np.float32)
+    for p in (1.0, 1.25, 2.0, 4.0, 10.0):
+        y = api.pow_spec(m, p)
+        ref = np.power(m.astype(np.float64), float(np.float32(p)))
+        ok = ref > 1e-36
+        assert np.max(np.abs(y[ok] - ref[ok]) / ref[ok]) <= 1e-5, p
+        assert np.all(np.diff(api.pow_spec(np.sort(m), p)) >= 0)
+    assert np.array_equal(api.pow_spec(np.array([0.0, 1.0, 0.5, 0.25], np.float32), 2.0),
+                          np.array([0.0, 1.0, 0.25, 0.0625], np.float32))
+    assert api.pow_spec(np.float32(1e-30), 10.0) == 0.0  # below 2^-125: flushed to zero by definition
+
+
+def pin_exponent_variant(api):
+    """Remark 3: the selection metric |a|^y * tanh(|1+Delta|/mu).  Its ranking, computed in binary64 from the
+    definition, must be the oracle's mask on inputs without near-ties; y = 1 is Algorithm 2 itself."""
+    rng = np.random.default_rng(17)
+    d, kp, mu, w = 64, 20, 2.0, 0.5
+    for y in (0.25, 0.5, 0.8):
+        for trial in range(5):
+            g = (rng.permutation(d) + 1.0).astype(np.float32) * rng.choice([-1.0, 1.0], size=d).astype(np.float32)
+            eps = np.zeros(d, np.float32)
+            pidx = np.sort(rng.choice(d, size=kp, replace=False)).astype(np.int32)
+            pval = (rng.integers(1, 60, size=kp) * rng.choice([-1.0, 1.0], size=kp)).astype(np.float32)
+            gprev = np.zeros(d, np.float32)
+            gprev[pidx] = rng.integers(-40, 40, size=kp).astype(np.float32)
+            a = g.astype(np.float64)
+            metric = np.abs(a) ** y
+            delta = (gprev[pidx].astype(np.float64) - w * pval.astype(np.float64)) / (w * a[pidx])
+            metric[pidx] *= np.tanh(np.abs(1.0 + delta) / mu)
+            order = np.argsort(-metric, kind="stable")
+            k = 16
+            # only the boundary between the k-th and the (k+1)-th matters for the mask; a near-tie there
+            # could fall either way in binary32: skip such a draw
+            if metric[order[k - 1]] - metric[order[k]] < 1e-3 * metric[order[k - 1]]:
+                continue
+            checked = locals().get("checked", 0) + 1
+            e = eps.copy()
+            idx, val = api.worker_step(g, e, k, pidx, pval, gprev, mu, w, 0, y)
+            assert np.array_equal(idx, np.sort(order[:k]).astype(np.int32)), (y, trial)
+            assert np.array_equal(val, g[idx])
+    assert checked >= 10
+    # y = 1 is the unmodified algorithm
+    g = rng.standard_normal(200).astype(np.float32)
+    pidx = np.arange(0, 200, 7, dtype=np.int32)
+    pval = rng.standard_normal(pidx.size).astype(np.float32)
+    gprev = rng.standard_normal(200).astype(np.float32)
+    a1 = api.scores(g, np.zeros(200, np.float32), pidx, pval, gprev, 4.0, 0.25, 1.0)[1]
+    a2 = api.scores(g, np.zeros(200, np.float32), pidx, pval, gprev, 4.0, 0.25)[1]
+    assert np.array_equal(a1, a2)
+    # off the previous support the score stays |a| for every y
+    s = api.scores(g, np.zeros(200, np.float32), pidx, pval, gprev, 4.0, 0.25, 0.5)[1]
+    off = np.setdiff1d(np.arange(200), pidx)
+    assert np.array_equal(s[off], np.abs(g[off]))
+    with np.testing.assert_raises(ValueError):
+        api.worker_step(g, np.zeros(200, np.float32), 5, None, None, None, 4.0, 0.25, 0, 1.5)
+
+
 def pin_model_update(api):
     """theta' = theta - eta*g with the product rounded first; entries with g = 0 keep their bits (also -0)."""
     theta = np.array([1.0, -0.0, 0.5, 2.0, 1.0], np.float32)
@@ -337,5 +395,5 @@ def pin_mask_certificate(api):
 
 ALL_PINS = [pin_tanh, pin_bruteforce_selector, pin_dense_passthrough, pin_reduces_to_topk,
             pin_error_feedback_identity, pin_toy_example, pin_table1_iteration1, pin_distortion_cases,
-            pin_regularised_ranking, pin_aggregation, pin_model_update, pin_bf16_gradients, pin_select_modes_agree,
+            pin_regularised_ranking, pin_aggregation, pin_pow, pin_exponent_variant, pin_model_update, pin_bf16_gradients, pin_select_modes_agree,
             pin_mask_certificate]

@@ -15,13 +15,13 @@ def bits(x):
 
 
 def run_parity(rounds, d, N, k, mu, omega=None, flags=0, check_eps=True, select_mode=0, threads=4,
-               reset_after=None, expect_dense=None):
+               reset_after=None, expect_dense=None, y=1.0):
     """rounds: iterable of torch tensors [N, ld] (CPU or CUDA, float32 or bfloat16).
     Returns the library's stats after the last round."""
     rounds = iter(rounds)
     first = next(rounds)
-    lib = RegTopK(d, N, k, mu=mu, omega=omega, grad_dtype=first.dtype, flags=flags)
-    ora = OracleRegTopK(d, N, k, mu, omega=omega, select_mode=select_mode, threads=threads)
+    lib = RegTopK(d, N, k, mu=mu, omega=omega, grad_dtype=first.dtype, flags=flags, y=y)
+    ora = OracleRegTopK(d, N, k, mu, omega=omega, select_mode=select_mode, threads=threads, y=y)
     t = 0
     g = first
     while g is not None:

@@ -57,6 +57,8 @@ def test_invalid_omega_and_dtype_rejected():
     assert binding.workspace_bytes(10, 2, 1, omega=[0.5, float("inf")]) == 0
     assert binding.workspace_bytes(10, 2, 1, grad_dtype=7) == 0
     assert binding.workspace_bytes(10, 2, 1, omega=[0.5, 0.5]) > 0
+    assert binding.workspace_bytes(10, 2, 1, y=0.5) > 0 and binding.workspace_bytes(10, 2, 1, y=0.0) > 0
+    assert binding.workspace_bytes(10, 2, 1, y=1.5) == 0 and binding.workspace_bytes(10, 2, 1, y=-0.5) == 0
 
 
 def test_null_context_calls(lib):

@@ -39,6 +39,16 @@ def test_mu_sweep(mu):
     run_parity(gauss_rounds(4, 50_001, 5, seed=3), 50_001, 4, 500, mu)
 
 
+@pytest.mark.parametrize("y", [0.25, 0.5, 0.9])
+def test_exponent_variant(y):
+    """Remark 3: selection metric |a|^y * regulariser."""
+    run_parity(gauss_rounds(4, 60_001, 6, seed=23), 60_001, 4, 600, 2.0, y=y)
+    w = synth.workload("resnet18", scale_to=200_000)
+    s = synth.GradientStream(w, device="cpu", seed=5, pad_to=8)
+    run_parity((s.next() for _ in range(5)), w.d, w.N, w.k_values()[1], w.mu, y=y,
+               flags=binding.FLAG_FORCE_DENSE_SELECT if y == 0.5 else 0)
+
+
 def test_custom_weights():
     run_parity(gauss_rounds(3, 30_000, 4, seed=5), 30_000, 3, 300, 4.0, omega=[0.3, 0.5, 0.2])
 

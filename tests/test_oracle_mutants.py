@@ -33,6 +33,10 @@ MUTANTS = [
     ("aggregate_no_weight", "float t = omega[n] * val[n * k + i];", "float t = val[n * k + i];"),
     ("aggregate_overwrites", "g_out[j] = g_out[j] + t;", "g_out[j] = t;"),
     ("aggregate_reverse_order", "for (int32_t n = 0; n < N; ++n) {", "for (int32_t n = N - 1; n >= 0; --n) {"),
+    ("exponent_not_inverted", "if (y != 1.0f) m = regtopk_oracle_pow(m, 1.0f / y);", "if (y != 1.0f) m = regtopk_oracle_pow(m, y);"),
+    ("exponent_ignored", "if (y != 1.0f) m = regtopk_oracle_pow(m, 1.0f / y);", ";"),
+    ("pow_log_sign", "float s = (f - 1.0f) / (f + 1.0f);", "float s = (1.0f - f) / (f + 1.0f);"),
+    ("pow_drops_exponent_part", "float L = static_cast<float>(e) + log2f;", "float L = log2f;"),
     ("update_adds", "theta[j] = theta[j] - step;", "theta[j] = theta[j] + step;"),
     ("update_ignores_eta", "float step = eta * g[j];", "float step = g[j];"),
     ("tanh_inverted", "return (1.0f - t) / (1.0f + t);", "return (1.0f + t) / (1.0f - t);"),
