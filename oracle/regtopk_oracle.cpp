@@ -30,8 +30,8 @@
 // Pins (tests/test_oracle_*.py): brute force over all subsets on tiny inputs; k = d pass-through;
 // round 0 / mu = 0 / mu -> 0 against an independent Top-k with error feedback; the error-feedback
 // identity; the toy logistic example (Delta = -1 exactly); the printed iteration-1 column of the
-// paper's low-dimensional table; hand-worked distortion examples; tanh against binary64 tanh;
-// aggregation against hand sums.  Multi-round trajectories on the paper's own data cannot be pinned
+// paper's low-dimensional table; hand-worked distortion examples; tanh and pow against binary64;
+// the exponent variant against its binary64 ranking; aggregation and the model update against hand sums.  Multi-round trajectories on the paper's own data cannot be pinned
 // (its data and seeds are not published): "parity unpinned" for those curves only.
 
 #include <algorithm>

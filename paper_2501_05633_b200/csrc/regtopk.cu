@@ -737,6 +737,7 @@ struct PostArgs {
   float* cur_val;
   int use_marks;  // previous support carries regularised scores (round >= 1, mu > 0)
   int has_stale;  // mask_new holds an old mask (round >= 2)
+  int pair_mode;  // many pairs: emit (index, value) as one store into the B list; k_unzip follows
 };
 
 __device__ __forceinline__ u32 warp_reserve_global(bool pred, u32* counter) {
@@ -1137,13 +1138,46 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
         if (word & bm) {
           const u32 r = s_segbase[(idx >> 8) / (u32)seg_units] + qp[q] + before + __popc(word & (bm - 1u));
           eps_row[idx] = 0.0f;  // a - a
-          p.out_idx[obase + r] = (int32_t)idx;
-          p.out_val[obase + r] = vv[q];
-          p.cur_idx[obase + r] = (int32_t)idx;
-          p.cur_val[obase + r] = vv[q];
+          if (p.pair_mode) {
+            // many pairs: one 8-byte store at the (random) rank instead of four 4-byte ones; k_unzip
+            // spreads the pairs over the four output arrays with sequential accesses afterwards
+            reinterpret_cast<uint2*>(B)[r] = make_uint2(idx, __float_as_uint(vv[q]));
+          } else {
+            p.out_idx[obase + r] = (int32_t)idx;
+            p.out_val[obase + r] = vv[q];
+            p.cur_idx[obase + r] = (int32_t)idx;
+            p.cur_val[obase + r] = vv[q];
+          }
         }
       }
     }
+  }
+}
+
+// After k_post in pair mode: (index, value) pairs, in rank order in the workers' B lists, go to the
+// caller's arrays and to the library's own copy.
+struct UnzipArgs {
+  const u64* candB;
+  int64_t stride;
+  int64_t k;
+  int N;
+  int32_t* out_idx;
+  float* out_val;
+  int32_t* cur_idx;
+  float* cur_val;
+};
+
+__global__ void __launch_bounds__(256) k_unzip(UnzipArgs p) {
+  grid_dependency_begin();
+  const int n = blockIdx.y;
+  const uint2* pairs = reinterpret_cast<const uint2*>(p.candB + (size_t)n * p.stride);
+  const size_t obase = (size_t)n * p.k;
+  for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < p.k; r += (int64_t)gridDim.x * blockDim.x) {
+    const uint2 v = __ldcs(pairs + r);
+    p.out_idx[obase + r] = (int32_t)v.x;
+    p.cur_idx[obase + r] = (int32_t)v.x;
+    p.out_val[obase + r] = __uint_as_float(v.y);
+    p.cur_val[obase + r] = __uint_as_float(v.y);
   }
 }
 
@@ -1635,6 +1669,7 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   pa.out_idx = out_idx; pa.out_val = out_val;
   pa.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); pa.cur_val = at<float>(c, L.off_val[c->cur]);
   pa.use_marks = use_marks; pa.has_stale = c->round >= 2;
+  pa.pair_mode = c->k * (int64_t)c->N >= 262144;
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[2];
   post_config(&cfg, attr, c->N, c->cluster, kBlockPost, c->stream);
@@ -1642,6 +1677,20 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   c->launches++;
   if (le != cudaSuccess) return note_cuda(c, le);
   if ((rc = note_cuda(c, cudaGetLastError()))) return rc;
+  if (pa.pair_mode) {
+    UnzipArgs ua;
+    ua.candB = pa.candB; ua.stride = L.stride; ua.k = c->k; ua.N = c->N;
+    ua.out_idx = out_idx; ua.out_val = out_val; ua.cur_idx = pa.cur_idx; ua.cur_val = pa.cur_val;
+    int64_t bx = (c->k + 255) / 256;
+    const int64_t cap_x = ((int64_t)c->num_sms * 16 + c->N - 1) / c->N;
+    if (bx > cap_x) bx = cap_x;
+    cudaLaunchConfig_t ucfg;
+    cudaLaunchAttribute uattr[2];
+    launch_config(&ucfg, uattr, (unsigned)bx, 1, 256, 0, c->stream);
+    ucfg.gridDim = dim3((unsigned)bx, (unsigned)c->N, 1);
+    cudaLaunchKernelEx(&ucfg, k_unzip, ua);
+    if ((rc = after_launch(c))) return rc;
+  }
 
   c->stepped = 1;
   return REGTOPK_OK;
