@@ -480,8 +480,9 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
 
 // ---------------------------------------------------------------------------------------------
 // k_stream: a = eps + g for all workers, in place; candidates appended.  Persistent grid, one
-// warp per 512-element chunk, chunks dealt round-robin so that neighbouring warps read
-// neighbouring memory.  12 (fp32) or 10 (bf16) bytes of HBM traffic per coordinate.
+// warp per chunk of 512 or 1024 elements (see StreamShape), chunks dealt round-robin so that
+// neighbouring warps read neighbouring memory.  12 (fp32) or 10 (bf16) bytes of HBM traffic per
+// coordinate.
 // ---------------------------------------------------------------------------------------------
 struct StreamArgs {
   const void* grads;
@@ -691,7 +692,7 @@ __global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC>::kBlock
 
 // ---------------------------------------------------------------------------------------------
 // k_post: one thread-block cluster per worker.  The cluster's blocks meet only at the hardware
-// cluster barrier; what they exchange (histograms, list lengths, per-block totals) goes through
+// cluster barrier; what they exchange (histograms, list lengths, segment totals) goes through
 // global memory, which the barrier's release/acquire makes visible.  Every block of a cluster
 // reaches every barrier: all branches that contain one depend only on values that are the same in
 // all blocks of the cluster.
