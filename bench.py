@@ -42,6 +42,9 @@ def parse():
     ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--api", default="plain", choices=["plain", "inplace"],
+                    help="inplace: the step is the caller's accumulate (torch add_ into the library's rows) + "
+                         "regtopk_worker_step_inplace + regtopk_aggregate; the library's share is reported beside it")
     return ap.parse_args()
 
 
@@ -219,8 +222,15 @@ def main():
     out_idx = torch.empty((w.N, k), dtype=torch.int32, device=dev)
     out_val = torch.empty((w.N, k), dtype=torch.float32, device=dev)
 
+    inplace = args.api == "inplace"
+    acc = lib.accumulator() if inplace else None
+
     def step(i):
-        lib.worker_step(ring[i % ring_n], out_idx, out_val)
+        if inplace:
+            acc.add_(ring[i % ring_n][:, : w.d])  # stands in for a backward pass that accumulates
+            lib.worker_step_inplace(out_idx, out_val)
+        else:
+            lib.worker_step(ring[i % ring_n], out_idx, out_val)
         lib.aggregate()
 
     def barrier():
@@ -261,9 +271,21 @@ def main():
     ms_prof = p0.elapsed_time(p1)
     kern_ms, calls = lib.profile_read()
     lib.profile_enable(False)
+    lib_only_ms = None
+    if inplace:  # the library's calls alone, one event pair per step
+        nlib = min(args.steps, 200)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(nlib)]
+        for i, (a0, a1) in enumerate(evs):
+            acc.add_(ring[i % ring_n][:, : w.d])
+            a0.record()
+            lib.worker_step_inplace(out_idx, out_val)
+            lib.aggregate()
+            a1.record()
+        torch.cuda.synchronize()
+        lib_only_ms = sum(a0.elapsed_time(a1) for a0, a1 in evs) / nlib
     # ---- end to end through host buffers ----
     e2e_s = float("nan")
-    if args.e2e_steps > 0:
+    if args.e2e_steps > 0 and not inplace:
         h_g = [ring[i].cpu().pin_memory() for i in range(min(2, ring_n))]
         h_idx = torch.empty((w.N, k), dtype=torch.int32).pin_memory()
         h_val = torch.empty((w.N, k), dtype=torch.float32).pin_memory()
@@ -285,8 +307,9 @@ def main():
         value = world * coords * args.steps / (ms_all * 1e-3) / 1e9
         peak, peak_kind = measured_peak()
         alg_bytes = coords * (bpe + 8)
+        kern_alg_bytes = coords * 4 if inplace else alg_bytes  # in place, the library only reads the rows
         kern_avg_ms = kern_ms / max(1, calls)
-        achieved = alg_bytes / (kern_avg_ms * 1e-3) / 1e9
+        achieved = kern_alg_bytes / (kern_avg_ms * 1e-3) / 1e9
         step_gbs = alg_bytes / (ms_all / args.steps * 1e-3) / 1e9
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -301,14 +324,18 @@ def main():
                        "candidates_last": stats_end["candidates_last"],
                        "ms_per_step_with_kernel_events": ms_prof / nprof},
             "clocks": clocks,
-            "e2e": {"value": (world * coords * args.e2e_steps / e2e_all / 1e9) if args.e2e_steps > 0 else None, "unit": UNIT,
+            "e2e": {"value": (world * coords * args.e2e_steps / e2e_all / 1e9) if (args.e2e_steps > 0 and not inplace) else None, "unit": UNIT,
                     "h2d_bytes_per_step": w.N * stream.ld * bpe, "d2h_bytes_per_step": 2 * w.N * k * 4 + w.d * 4},
             "gpu_launches": launches,
             "roofline": {"bound": "hbm", "kernel": "k_stream", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "traffic": NCU_STREAM_TRAFFIC.get(w.name) if w.grad_dtype == "f32" else None,
-                         "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": kern_avg_ms},
+                         "algorithmic_bytes_per_launch": kern_alg_bytes, "avg_launch_ms": kern_avg_ms},
         }
+        if inplace:
+            line["config"]["api"] = ("accumulate in place: ms_per_step includes the caller's torch add_ of the gradients "
+                                     "into the library's rows; ms_library_only is worker_step_inplace + aggregate alone")
+            line["config"]["ms_library_only"] = lib_only_ms
         if world == 1 and not args.no_cpu_baseline:
             del ring
             torch.cuda.empty_cache()

@@ -90,6 +90,21 @@ int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const reg
 int regtopk_worker_step(regtopk_ctx* ctx, const void* grads, int64_t grad_ld, int32_t* out_idx,
                         float* out_val);
 
+/* Accumulate-in-place form of the same round, for callers whose gradient computation can add into a
+ * buffer (a backward pass that accumulates): Algorithm 2 step 6, a_n^t = eps_n^t + g_n^t, is then the
+ * caller's own addition, and the library never reads a separate gradient array nor rewrites the
+ * accumulator: 4 bytes of memory traffic per coordinate and worker instead of 12.
+ *   regtopk_accumulator gives the device pointer to the library's rows ([N][*ld] binary32, row n at
+ *   *dev_ptr + n * *ld, *ld >= d).  Between rounds row n holds eps_n^t.  Before
+ *   regtopk_worker_step_inplace the caller, on the context's stream (or ordered before it), adds
+ *   g_n^t[j] to element j of row n for j < d, in binary32 with a single round-to-nearest addition
+ *   per element; elements [d, *ld) must stay 0.  The context's grad_dtype is not used by this form.
+ *   regtopk_worker_step_inplace then does what regtopk_worker_step does from its accumulate step on
+ *   (steps 7-12), with the same outputs, errors and call order; the two forms may be mixed from round
+ *   to round, and the results are bit-identical to regtopk_worker_step given the same gradients. */
+int regtopk_accumulator(regtopk_ctx* ctx, float** dev_ptr, int64_t* ld);
+int regtopk_worker_step_inplace(regtopk_ctx* ctx, int32_t* out_idx, float* out_val);
+
 /* Server side of the round (Section 2.2): g^t = sum_n omega_n * ghat_n^t, workers added in the order
  * n = 0..N-1 with each product rounded before its addition, then the state roll for round t+1 (the
  * pairs just sent become the previous mask and a^{t} on it, g^t becomes g^{t-1}).

@@ -27,7 +27,7 @@ EXPORTS = [
     "regtopk_global_gradient", "regtopk_state_reset", "regtopk_round_host", "regtopk_status",
     "regtopk_get_stats", "regtopk_profile_enable", "regtopk_profile_read", "regtopk_debug_residual",
     "regtopk_destroy", "regtopk_strerror", "regtopk_aggregate_pairs_static", "regtopk_aggregate_update", "regtopk_state_bytes",
-    "regtopk_state_export", "regtopk_state_import",
+    "regtopk_state_export", "regtopk_state_import", "regtopk_accumulator", "regtopk_worker_step_inplace",
 ]
 
 
@@ -103,6 +103,10 @@ def load_library():
     L.regtopk_profile_enable.argtypes = [vp, ctypes.c_int]
     L.regtopk_profile_read.restype = ctypes.c_int
     L.regtopk_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
+    L.regtopk_accumulator.restype = ctypes.c_int
+    L.regtopk_accumulator.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i64)]
+    L.regtopk_worker_step_inplace.restype = ctypes.c_int
+    L.regtopk_worker_step_inplace.argtypes = [vp, vp, vp]
     L.regtopk_debug_residual.restype = ctypes.c_int
     L.regtopk_debug_residual.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(i64)]
     L.regtopk_destroy.restype = ctypes.c_int
@@ -237,6 +241,25 @@ class RegTopK:
             out_val = torch.empty((self.N, self.k), dtype=torch.float32, device=self.device)
         _check(self.L.regtopk_worker_step(self.ctx, grads.data_ptr(), ld, out_idx.data_ptr(),
                                           out_val.data_ptr()), "regtopk_worker_step")
+        return out_idx, out_val
+
+    def accumulator(self) -> torch.Tensor:
+        """Writable view [N, d] of the library's accumulator rows: add each worker's gradient into its row
+        (binary32, one addition per element), then call worker_step_inplace()."""
+        ptr, ld = ctypes.c_void_p(), ctypes.c_int64()
+        _check(self.L.regtopk_accumulator(self.ctx, ctypes.byref(ptr), ctypes.byref(ld)), "regtopk_accumulator")
+        off = ptr.value - self.workspace.data_ptr()
+        full = self.workspace[off: off + 4 * self.N * ld.value].view(torch.float32).view(self.N, ld.value)
+        return full[:, : self.d]
+
+    def worker_step_inplace(self, out_idx: Optional[torch.Tensor] = None,
+                            out_val: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+        if out_idx is None:
+            out_idx = torch.empty((self.N, self.k), dtype=torch.int32, device=self.device)
+        if out_val is None:
+            out_val = torch.empty((self.N, self.k), dtype=torch.float32, device=self.device)
+        _check(self.L.regtopk_worker_step_inplace(self.ctx, out_idx.data_ptr(), out_val.data_ptr()),
+               "regtopk_worker_step_inplace")
         return out_idx, out_val
 
     def aggregate(self, out: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -282,6 +282,7 @@ struct SampleArgs {
   float inv_y;              // 1/y of the exponent variant (1: Algorithm 2 as printed)
   u32* ovr_key;             // [N][k] out: score bits
   int share_override;       // the sampling blocks take a share of the override work too
+  int inplace;              // the caller has already added g into the rows of eps: a is read from there, grads is NULL
 };
 
 // Add a block's histogram to the cluster's in global memory (non-empty bins only).
@@ -313,14 +314,17 @@ __device__ __forceinline__ void override_scores(const SampleArgs& p, int64_t fir
     for (int q = 0; q < 4; ++q) {
       const bool in = t0 + q * nthreads < total;
       G[q] = in ? p.g_prev[j[q]] : 0.0f;
-      gr[q] = in ? load_grad<BF16>(static_cast<const char*>(p.grads) + (size_t)wn[q] * p.grad_ld * (BF16 ? 2 : 4), j[q]) : 0.0f;
+      if (p.inplace)
+        gr[q] = in ? p.eps[(size_t)wn[q] * p.ld + j[q]] : 0.0f;  // the residual there was +0: the row holds 0 + g
+      else
+        gr[q] = in ? load_grad<BF16>(static_cast<const char*>(p.grads) + (size_t)wn[q] * p.grad_ld * (BF16 ? 2 : 4), j[q]) : 0.0f;
     }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int64_t t = t0 + q * nthreads;
       if (t < total) {
         const float w = p.omega[wn[q]];
-        const float a = __fadd_rn(0.0f, gr[q]);
+        const float a = p.inplace ? gr[q] : __fadd_rn(0.0f, gr[q]);
         const float num = __fsub_rn(G[q], __fmul_rn(w, ap[q]));
         const float den = __fmul_rn(w, a);
         float m = 1.0f;
@@ -394,13 +398,13 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
       const int64_t j = q * 8 + (i & 7);
       ok[u] = i < nslots && j < p.d;
       e[u] = ok[u] ? eps_row[j] : 0.0f;
-      g[u] = ok[u] ? load_grad<BF16>(grow, j) : 0.0f;
+      g[u] = (ok[u] && !p.inplace) ? load_grad<BF16>(grow, j) : 0.0f;
     }
     for (int i = tid; i < kSamplePadded; i += blockDim.x) s_hist[i] = 0;  // while the loads are in flight
     __syncthreads();
 #pragma unroll
     for (int u = 0; u < 8; ++u)
-      if (ok[u]) atomicAdd(&s_hist[sample_slot((__float_as_uint(__fadd_rn(e[u], g[u])) & 0x7FFFFFFFu) >> kSampleShift)], 1u);
+      if (ok[u]) atomicAdd(&s_hist[sample_slot((__float_as_uint(p.inplace ? e[u] : __fadd_rn(e[u], g[u])) & 0x7FFFFFFFu) >> kSampleShift)], 1u);
   }
   __syncthreads();
   for (int i = tid; i < kSampleBins; i += blockDim.x) {
@@ -563,7 +567,10 @@ __device__ __forceinline__ void stream_flush(u64* list, u32& wcount, WorkerCtl* 
 #ifndef REGTOPK_STREAM_EPL_BF16
 #define REGTOPK_STREAM_EPL_BF16 8
 #endif
-template <bool BF16, bool VEC>
+#ifndef REGTOPK_STREAM_BLOCKS_INPLACE
+#define REGTOPK_STREAM_BLOCKS_INPLACE 3
+#endif
+template <bool BF16, bool VEC, bool INPLACE = false>
 struct StreamShape {
   static constexpr int kEpl = (BF16 && VEC) ? REGTOPK_STREAM_EPL_BF16 : 4;  // elements per lane and step
   static constexpr int kVec = kEpl / 4;                     // float4 vectors per lane and step
@@ -576,12 +583,15 @@ struct StreamShape {
 #ifndef REGTOPK_STREAM_BLOCKS_BF16
 #define REGTOPK_STREAM_BLOCKS_BF16 3
 #endif
-  static constexpr int kBlocksPerSm = (BF16 && VEC) ? REGTOPK_STREAM_BLOCKS_BF16 : (VEC ? REGTOPK_STREAM_BLOCKS_F32 : 2);
+  static constexpr int kBlocksPerSm = INPLACE ? REGTOPK_STREAM_BLOCKS_INPLACE
+                                      : (BF16 && VEC) ? REGTOPK_STREAM_BLOCKS_BF16 : (VEC ? REGTOPK_STREAM_BLOCKS_F32 : 2);
 };
 
-template <bool BF16, bool VEC>
-__global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC>::kBlocksPerSm) k_stream(StreamArgs p) {
-  typedef StreamShape<BF16, VEC> S;
+// INPLACE: the rows of eps already hold a = eps + g (the caller added its gradients there); nothing but
+// those rows is read and nothing is written back: 4 bytes of HBM traffic per coordinate.
+template <bool BF16, bool VEC, bool INPLACE>
+__global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC, INPLACE>::kBlocksPerSm) k_stream(StreamArgs p) {
+  typedef StreamShape<BF16, VEC, INPLACE> S;
   __shared__ u64 s_list[kStreamThreads / 32][kWarpList];
   grid_dependency_begin();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -615,7 +625,9 @@ __global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC>::kBlock
 #pragma unroll
       for (int v = 0; v < S::kVec; ++v)
         e[u][v] = __ldcs(reinterpret_cast<const float4*>(eps_row + j + 4 * v));  // rows are padded: in bounds
-      if (VEC && (full || j + S::kEpl - 1 < p.d)) {
+      if (INPLACE) {
+        // no gradient to load
+      } else if (VEC && (full || j + S::kEpl - 1 < p.d)) {
         if (BF16) {
           if (S::kEpl == 8) {  // eight bf16 in one 16-byte load
             const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(grow + j * 2));
@@ -654,12 +666,16 @@ __global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC>::kBlock
       for (int v = 0; v < S::kVec; ++v) {
         const int64_t j = base + u * S::kStep + lane * S::kEpl + 4 * v;
         float4 a;
-        a.x = __fadd_rn(e[u][v].x, g[u][v].x);
-        a.y = __fadd_rn(e[u][v].y, g[u][v].y);
-        a.z = __fadd_rn(e[u][v].z, g[u][v].z);
-        a.w = __fadd_rn(e[u][v].w, g[u][v].w);
-        __stcs(reinterpret_cast<float4*>(eps_row + j), a);  // padding receives 0 + 0; streaming store: the
-                                                            // accumulators should not push the small lists out of L2
+        if (INPLACE) {
+          a = e[u][v];
+        } else {
+          a.x = __fadd_rn(e[u][v].x, g[u][v].x);
+          a.y = __fadd_rn(e[u][v].y, g[u][v].y);
+          a.z = __fadd_rn(e[u][v].z, g[u][v].z);
+          a.w = __fadd_rn(e[u][v].w, g[u][v].w);
+          __stcs(reinterpret_cast<float4*>(eps_row + j), a);  // padding receives 0 + 0; streaming store: the
+                                                              // accumulators should not push the small lists out of L2
+        }
         const u32 k0 = __float_as_uint(a.x) & 0x7FFFFFFFu, k1 = __float_as_uint(a.y) & 0x7FFFFFFFu;
         const u32 k2 = __float_as_uint(a.z) & 0x7FFFFFFFu, k3 = __float_as_uint(a.w) & 0x7FFFFFFFu;
         const bool h0 = k0 >= cutoff && (full || j + 0 < p.d);
@@ -1429,7 +1445,7 @@ struct regtopk_ctx {
   int sticky;        // first CUDA error seen
   int num_sms;
   int cluster;       // blocks per worker in k_post
-  int stream_blocks[4];
+  int stream_blocks[5];
   int64_t launches;
   int profiling;
   int n_events;
@@ -1479,22 +1495,22 @@ void launch_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, unsigned 
   cfg->numAttrs = na;
 }
 
-template <bool BF16, bool VEC>
+template <bool BF16, bool VEC, bool INPLACE = false>
 void launch_stream(regtopk_ctx* c, const StreamArgs& a, int variant) {
   if (c->stream_blocks[variant] == 0) {
     int per_sm = 0;
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_stream<BF16, VEC>, kStreamThreads, 0);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_stream<BF16, VEC, INPLACE>, kStreamThreads, 0);
     if (per_sm < 1) per_sm = 1;
     c->stream_blocks[variant] = per_sm * c->num_sms;
   }
-  const int64_t chunk = StreamShape<BF16, VEC>::kChunk;
+  const int64_t chunk = StreamShape<BF16, VEC, INPLACE>::kChunk;
   const int64_t chunks = ((a.d + chunk - 1) / chunk) * a.N;
   int64_t blocks = (chunks + (kStreamThreads / 32) - 1) / (kStreamThreads / 32);
   if (blocks > c->stream_blocks[variant]) blocks = c->stream_blocks[variant];
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[2];
   launch_config(&cfg, attr, (unsigned)blocks, 1, kStreamThreads, 0, c->stream);
-  cudaLaunchKernelEx(&cfg, k_stream<BF16, VEC>, a);
+  cudaLaunchKernelEx(&cfg, k_stream<BF16, VEC, INPLACE>, a);
 }
 
 void post_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int N, int cluster, int threads,
@@ -1604,12 +1620,19 @@ int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const reg
   return REGTOPK_OK;
 }
 
-int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_idx,
-                        float* out_val) {
-  if (!c || !grads || !out_idx || !out_val || grad_ld < c->d) return REGTOPK_ERR_INVALID_ARG;
+}  // extern "C"
+
+namespace {
+// One round of all workers.  grads == NULL: the accumulator rows already hold a (regtopk_worker_step_inplace).
+int step_impl(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_idx, float* out_val) {
   if (c->stepped) return REGTOPK_ERR_SEQUENCE;
   const Layout& L = c->L;
-  const bool bf16 = c->grad_dtype == REGTOPK_GRAD_BF16;
+  const bool inplace = grads == nullptr;
+  if (inplace) {  // never dereferenced; keeps the row arithmetic of the sampling kernel on a real buffer
+    grads = at<float>(c, L.off_eps);
+    grad_ld = L.ld;
+  }
+  const bool bf16 = !inplace && c->grad_dtype == REGTOPK_GRAD_BF16;
   const bool has_prev = c->round >= 1;
   const bool use_marks = has_prev && c->mu > 0.0f;
   const int prev = c->cur ^ 1;
@@ -1629,6 +1652,7 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   sa.prev_idx = at<int32_t>(c, L.off_idx[prev]); sa.prev_val = at<float>(c, L.off_val[prev]);
   sa.omega = at<float>(c, L.off_omega); sa.mu = c->mu; sa.inv_y = c->inv_y; sa.ovr_key = at<u32>(c, L.off_ovr_key);
   sa.share_override = 0;
+  sa.inplace = inplace ? 1 : 0;
   sa.force_dense = (c->flags & REGTOPK_FLAG_FORCE_DENSE_SELECT) ? 1 : 0;
   {
     cudaLaunchConfig_t scfg;
@@ -1651,7 +1675,8 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
   st.marks = use_marks ? at<u32>(c, L.off_mask[prev]) : nullptr; st.W = L.W;
   const bool prof = c->profiling && c->n_events < kMaxProfile;
   if (prof) cudaEventRecord(c->ev0[c->n_events], c->stream);
-  if (bf16) { if (vec) launch_stream<true, true>(c, st, 3); else launch_stream<true, false>(c, st, 2); }
+  if (inplace) launch_stream<false, true, true>(c, st, 4);
+  else if (bf16) { if (vec) launch_stream<true, true>(c, st, 3); else launch_stream<true, false>(c, st, 2); }
   else { if (vec) launch_stream<false, true>(c, st, 1); else launch_stream<false, false>(c, st, 0); }
   if (prof) cudaEventRecord(c->ev1[c->n_events++], c->stream);
   if ((rc = after_launch(c))) return rc;
@@ -1695,6 +1720,27 @@ int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int3
 
   c->stepped = 1;
   return REGTOPK_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int regtopk_worker_step(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_idx,
+                        float* out_val) {
+  if (!c || !grads || !out_idx || !out_val || grad_ld < c->d) return REGTOPK_ERR_INVALID_ARG;
+  return step_impl(c, grads, grad_ld, out_idx, out_val);
+}
+
+int regtopk_accumulator(regtopk_ctx* c, float** dev_ptr, int64_t* ld) {
+  if (!c || !dev_ptr || !ld) return REGTOPK_ERR_INVALID_ARG;
+  *dev_ptr = at<float>(c, c->L.off_eps);
+  *ld = c->L.ld;
+  return REGTOPK_OK;
+}
+
+int regtopk_worker_step_inplace(regtopk_ctx* c, int32_t* out_idx, float* out_val) {
+  if (!c || !out_idx || !out_val) return REGTOPK_ERR_INVALID_ARG;
+  return step_impl(c, nullptr, 0, out_idx, out_val);
 }
 
 int regtopk_aggregate(regtopk_ctx* c, float* out_g) { return regtopk_aggregate_update(c, nullptr, 0.0f, out_g); }

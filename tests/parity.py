@@ -15,8 +15,9 @@ def bits(x):
 
 
 def run_parity(rounds, d, N, k, mu, omega=None, flags=0, check_eps=True, select_mode=0, threads=4,
-               reset_after=None, expect_dense=None, y=1.0):
+               reset_after=None, expect_dense=None, y=1.0, inplace=None):
     """rounds: iterable of torch tensors [N, ld] (CPU or CUDA, float32 or bfloat16).
+    inplace: None, or a function of the round number saying whether that round uses the accumulate-in-place calls.
     Returns the library's stats after the last round."""
     rounds = iter(rounds)
     first = next(rounds)
@@ -27,7 +28,12 @@ def run_parity(rounds, d, N, k, mu, omega=None, flags=0, check_eps=True, select_
     while g is not None:
         g_dev = g if g.is_cuda else g.cuda()
         g_cpu = g.cpu() if g.is_cuda else g
-        idx, val = lib.worker_step(g_dev)
+        if inplace is not None and inplace(t):
+            # accumulate-in-place form: the caller adds the gradients into the library's rows itself
+            lib.accumulator().add_(g_dev[:, :d].float())
+            idx, val = lib.worker_step_inplace()
+        else:
+            idx, val = lib.worker_step(g_dev)
         o_idx, o_val = ora.worker_step(to_oracle_view(g_cpu, d))
         lib.status()
         idx_h, val_h = idx.cpu().numpy(), val.cpu().numpy()

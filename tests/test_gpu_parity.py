@@ -188,6 +188,30 @@ def test_sample_underestimates_cutoff():
     run_parity(rounds, d, N, k, 4.0, expect_dense=True)
 
 
+# ---- accumulate-in-place calls: the caller adds g into the library's rows, the library only scans them ------
+@pytest.mark.parametrize("d,N,k", [(1, 1, 1), (7, 3, 7), (513, 3, 1), (4096, 8, 41), (65537, 2, 655),
+                                   (200003, 4, 2000), (200003, 2, 200003), (1_000_003, 2, 1000), (70_000, 150, 70)])
+@pytest.mark.parametrize("mu", [4.0, 0.0])
+def test_inplace_sizes(d, N, k, mu):
+    run_parity(gauss_rounds(N, d, 4, seed=d + N + 2), d, N, k, mu, inplace=lambda t: True)
+
+
+def test_inplace_mixed_with_plain_rounds_bf16_and_dense_path():
+    run_parity(gauss_rounds(3, 150_000, 6, seed=61), 150_000, 3, 1500, 4.0, inplace=lambda t: t % 2 == 1)
+    run_parity(gauss_rounds(2, 120_007, 4, seed=62, ld=120_008, dtype=torch.bfloat16), 120_007, 2, 1200, 4.0,
+               inplace=lambda t: t >= 2)
+    run_parity(gauss_rounds(3, 90_001, 4, seed=63), 90_001, 3, 900, 4.0, flags=binding.FLAG_FORCE_DENSE_SELECT,
+               expect_dense=True, inplace=lambda t: True)
+    run_parity(gauss_rounds(3, 80_000, 4, seed=64, quant=2), 80_000, 3, 800, 2.0, y=0.5, inplace=lambda t: True)
+
+
+def test_inplace_scaled_workload_long_run():
+    w = synth.workload("resnet18", scale_to=400_000)
+    s = synth.GradientStream(w, device="cpu", seed=33, pad_to=8)
+    st = run_parity((s.next() for _ in range(20)), w.d, w.N, w.k_values()[0], w.mu, threads=8, inplace=lambda t: True)
+    assert st["dense_select_workers"] == 0, st
+
+
 # ---- model-shaped workloads, scaled down (several tiles, ragged tail) ---------------------------------
 @pytest.mark.parametrize("name", ["resnet18", "resnet50", "gpt2", "flat1p3b"])
 def test_scaled_workloads(name):
