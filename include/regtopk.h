@@ -51,7 +51,9 @@ enum { REGTOPK_GRAD_F32 = 0, REGTOPK_GRAD_BF16 = 1 };
 /* flags of regtopk_params */
 enum {
   REGTOPK_FLAG_HOST_STAGING = 1,      /* reserve workspace for regtopk_round_host                          */
-  REGTOPK_FLAG_FORCE_DENSE_SELECT = 2 /* testing: skip the sampled cutoff, always take the dense exact path */
+  REGTOPK_FLAG_FORCE_DENSE_SELECT = 2, /* testing: skip the sampled cutoff, always take the dense exact path */
+  REGTOPK_FLAG_FORCE_WIDE_LISTS = 4    /* testing: handle the candidate lists the way large N*k is handled (separate
+                                          full-grid kernels, pairs unzipped afterwards) at any size; same results */
 };
 
 typedef struct {

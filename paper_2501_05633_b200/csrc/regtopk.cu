@@ -72,7 +72,11 @@ struct WorkerCtl {
   u32 bcount;       // length of the refinement list
   u32 acount;       // dense path: entries above the threshold gathered so far
   u32 n_valid;      // valid items seen by the select (diagnostics)
-  u32 pad;
+  u32 b1;           // wide mode: threshold bin, entries above it, and whether the row needs the dense
+  u32 above1;       //   exact path (written by k_wide_classify, read by k_post and k_wide_emit)
+  u32 go_dense;
+  u32 took_dense;   // wide mode: the dense path produced the winner list (written by k_post)
+  u32 pad[5];
 };
 
 struct GlobalCtl {
@@ -376,6 +380,8 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
       ctl->bcount = 0;
       ctl->acount = 0;
       ctl->n_valid = 0;
+    ctl->b1 = kFull; ctl->above1 = 0; ctl->go_dense = 0; ctl->took_dense = 0;
+      ctl->b1 = kFull; ctl->above1 = 0; ctl->go_dense = 0; ctl->took_dense = 0;
     }
     return;
   }
@@ -479,6 +485,7 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
     ctl->bcount = 0;
     ctl->acount = 0;
     ctl->n_valid = 0;
+    ctl->b1 = kFull; ctl->above1 = 0; ctl->go_dense = 0; ctl->took_dense = 0;
   }
 }
 
@@ -755,6 +762,7 @@ struct PostArgs {
   int use_marks;  // previous support carries regularised scores (round >= 1, mu > 0)
   int has_stale;  // mask_new holds an old mask (round >= 2)
   int pair_mode;  // many pairs: emit (index, value) as one store into the B list; k_unzip follows
+  int wide;       // k_post runs between the wide kernels: refinement or dense path only
 };
 
 __device__ __forceinline__ u32 warp_reserve_global(bool pred, u32* counter) {
@@ -867,6 +875,184 @@ __device__ __forceinline__ u32 popc4(const uint4& v) {
   return (u32)(__popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w));
 }
 
+// ---- pieces of the selection, shared by k_post (one cluster per worker) and the wide kernels (the whole
+//      grid split over the workers; used when N*k is large).  first_t / stride_t: this thread's index
+//      among, and the number of, the threads that work on worker n's row. ----
+
+// One sweep over the lists, a single wave of coalesced loads per step:
+//   (a) the mask buffer of this round still holds the mask of two rounds ago: clear those words;
+//   (b) the override scores (written by k_sample_cutoff's override clusters) that reach the cutoff
+//       become composites and enter the histogram;
+//   (c) the candidates (k_stream already dropped those on the previous support) enter it too.
+__device__ __forceinline__ void post_sweep(const PostArgs& p, int n, u32 first_t, u32 stride_t, bool dense,
+                                           u32 ncand, u32 cutoff, u32 bshift, u32* s_hist) {
+  const u32 k = (u32)p.k;
+  const size_t obase = (size_t)n * p.k;
+  const u64* A = p.candA + (size_t)n * p.stride;
+  u64* O = p.ovr_comp + obase;
+  const u32* okey = p.ovr_key + obase;
+  const int32_t* prev_idx = p.prev_idx + obase;
+  u32* mask = p.mask_new + (size_t)n * p.W;
+  const u32 span = !dense && ncand > k ? ncand : k;
+  constexpr int kP0 = 8;  // items per thread in flight
+  for (u32 i0 = first_t; i0 < span; i0 += kP0 * stride_t) {
+    int32_t stale[kP0], j[kP0];
+    u32 key[kP0];
+    u64 c[kP0];
+#pragma unroll
+    for (int q = 0; q < kP0; ++q) {
+      const u32 i = i0 + q * stride_t;
+      const bool in_k = i < k;
+      stale[q] = (in_k && p.has_stale) ? p.cur_idx[obase + i] : -1;
+      j[q] = (in_k && p.use_marks) ? prev_idx[i] : -1;
+      key[q] = (in_k && p.use_marks) ? okey[i] : 0u;
+      c[q] = (!dense && i < ncand) ? A[i] : 0ull;
+    }
+#pragma unroll
+    for (int q = 0; q < kP0; ++q) {
+      const u32 i = i0 + q * stride_t;
+      if (stale[q] >= 0) mask[(u32)stale[q] >> 5] = 0u;
+      if (j[q] >= 0) {
+        const u64 oc = key[q] >= cutoff ? make_composite(key[q], (u32)j[q]) : 0ull;
+        O[i] = oc;
+        if (!dense && oc) atomicAdd(&s_hist[select_bin(key[q], cutoff, bshift)], 1u);
+      }
+      if (c[q]) atomicAdd(&s_hist[select_bin((u32)(c[q] >> 32), cutoff, bshift)], 1u);
+    }
+  }
+}
+
+// Classify candidates and overrides (one item list, eight loads per thread in flight): above the threshold
+// bin -> winner; inside it -> refinement list.  Whole warps must call it.
+__device__ __forceinline__ void post_classify(const PostArgs& p, int n, u32 first_t, u32 stride_t, u32 ncand,
+                                              u32 novr, u32 cutoff, u32 bshift, u32 b1) {
+  const u64* A = p.candA + (size_t)n * p.stride;
+  u64* B = p.candB + (size_t)n * p.stride;
+  const u64* O = p.ovr_comp + (size_t)n * p.k;
+  u32* mask = p.mask_new + (size_t)n * p.W;
+  WorkerCtl* ctl = p.ctl + n;
+  const u32 total_items = ncand + novr;
+  const u32 iters = (total_items + 8 * stride_t - 1) / (8 * stride_t);
+  for (u32 it = 0; it < iters; ++it) {
+    u64 c[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const u32 t = (it * 8 + q) * stride_t + first_t;
+      c[q] = t < ncand ? __ldcg(A + t) : (t < total_items ? __ldcg(O + (t - ncand)) : 0ull);
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const u32 bin = c[q] ? select_bin((u32)(c[q] >> 32), cutoff, bshift) : 0u;
+      if (c[q] && bin > b1) set_winner(mask, composite_idx(c[q]));
+      const bool inbin = c[q] && bin == b1;
+      const u32 pos = warp_reserve_global(inbin, &ctl->bcount);
+      if (inbin) B[pos] = c[q];
+    }
+  }
+}
+
+// One warp: per quad (four mask words, 128 coordinates) of segment `seg`, the mask bits before it inside
+// the segment; the segment's total.  Segments are runs of seg_units 8-word units of the mask row.
+__device__ __forceinline__ void post_prefix_segment(const PostArgs& p, int n, u32 seg, int64_t seg_units, int lane) {
+  const int64_t U = p.W >> 3;
+  const uint4* quads = reinterpret_cast<const uint4*>(p.mask_new + (size_t)n * p.W);
+  u32* qpre = p.qprefix + (size_t)n * (p.W >> 2);
+  const int64_t wu0 = (int64_t)seg * seg_units < U ? (int64_t)seg * seg_units : U;
+  const int64_t wu1 = wu0 + seg_units < U ? wu0 + seg_units : U;
+  u32 running = 0;
+  for (int64_t ub = wu0; ub < wu1; ub += 128) {  // four rows of 32 units per step
+    uint4 x[4], y[4];
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      const int64_t u = ub + it * 32 + lane;
+      x[it] = u < wu1 ? __ldcg(quads + 2 * u) : make_uint4(0, 0, 0, 0);
+      y[it] = u < wu1 ? __ldcg(quads + 2 * u + 1) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      const u32 cx = popc4(x[it]), c = cx + popc4(y[it]);
+      u32 inc = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const u32 t = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += t;
+      }
+      const int64_t u = ub + it * 32 + lane;
+      const u32 pre = running + inc - c;
+      if (u < wu1) *reinterpret_cast<uint2*>(qpre + 2 * u) = make_uint2(pre, pre + cx);
+      running += __shfl_sync(kFull, inc, 31);
+    }
+  }
+  if (lane == 0) p.segtot[(size_t)n * kMaxSegments + seg] = running;
+}
+
+// Every item whose mask bit is set looks its rank up (segment base + quad prefix + bits before it in
+// the quad), writes its (index, value) pair there and zeroes its residual.  Normal path: candidates and
+// overrides as one item list; dense path: its k winners, nothing else.  Items below the threshold bin
+// cannot have won and are skipped without touching memory.
+__device__ __forceinline__ void post_emit(const PostArgs& p, int n, u32 first_t, u32 stride_t, u32 ncand, u32 novr,
+                                          bool took_dense, u32 cutoff, u32 bshift, u32 b1, const u32* s_segbase,
+                                          int64_t seg_units) {
+  const u32 k = (u32)p.k;
+  const size_t obase = (size_t)n * p.k;
+  const u64* A = p.candA + (size_t)n * p.stride;
+  u64* B = p.candB + (size_t)n * p.stride;
+  const u64* O = p.ovr_comp + obase;
+  float* eps_row = p.eps + (size_t)n * p.ld;
+  const uint4* quads = reinterpret_cast<const uint4*>(p.mask_new + (size_t)n * p.W);
+  const u32* qpre = p.qprefix + (size_t)n * (p.W >> 2);
+  const u32 nA = took_dense ? k : ncand;
+  const u32 total_items = nA + (took_dense ? 0u : novr);
+  for (u32 t0 = first_t; t0 < total_items; t0 += 4 * stride_t) {
+    u64 c[4];
+    uint4 qw[4];
+    u32 qp[4];
+    float vv[4];
+    bool live[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const u32 t = t0 + q * stride_t;
+      c[q] = t < nA ? __ldcg(A + t) : (t < total_items ? __ldcg(O + (t - nA)) : 0ull);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const u32 idx = composite_idx(c[q]);
+      live[q] = c[q] != 0ull && (took_dense || select_bin((u32)(c[q] >> 32), cutoff, bshift) >= b1);
+      qw[q] = live[q] ? __ldcg(quads + (idx >> 7)) : make_uint4(0, 0, 0, 0);
+      qp[q] = live[q] ? __ldcg(qpre + (idx >> 7)) : 0u;
+      vv[q] = live[q] ? eps_row[idx] : 0.0f;
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (!live[q]) continue;
+      const u32 idx = composite_idx(c[q]);
+      const u32 w[4] = {qw[q].x, qw[q].y, qw[q].z, qw[q].w};
+      const u32 wsel = (idx >> 5) & 3u;
+      u32 before = 0, word = 0;
+#pragma unroll
+      for (int wi = 0; wi < 4; ++wi) {
+        if ((u32)wi < wsel) before += __popc(w[wi]);
+        if ((u32)wi == wsel) word = w[wi];
+      }
+      const u32 bm = 1u << (idx & 31);
+      if (word & bm) {
+        const u32 r = s_segbase[(idx >> 8) / (u32)seg_units] + qp[q] + before + __popc(word & (bm - 1u));
+        eps_row[idx] = 0.0f;  // a - a
+        if (p.pair_mode) {
+          // many pairs: one 8-byte store at the (random) rank instead of four 4-byte ones; k_unzip
+          // spreads the pairs over the four output arrays with sequential accesses afterwards
+          reinterpret_cast<uint2*>(B)[r] = make_uint2(idx, __float_as_uint(vv[q]));
+        } else {
+          p.out_idx[obase + r] = (int32_t)idx;
+          p.out_val[obase + r] = vv[q];
+          p.cur_idx[obase + r] = (int32_t)idx;
+          p.cur_val[obase + r] = vv[q];
+        }
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs p) {
   __shared__ __align__(16) PostShared sh;
   grid_dependency_begin();
@@ -883,14 +1069,9 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
   const u32 k = (u32)p.k;
   u64* A = p.candA + (size_t)n * p.stride;
   u64* B = p.candB + (size_t)n * p.stride;
-  u64* O = p.ovr_comp + (size_t)n * p.k;
-  u32* okey = p.ovr_key + (size_t)n * p.k;
-  const int32_t* prev_idx = p.prev_idx + (size_t)n * p.k;
   u32* mask = p.mask_new + (size_t)n * p.W;
   u32* ghist = p.ghist + (size_t)n * 4 * kBins;
   u32* btot = p.btot + (size_t)n * 2 * kMaxCluster;
-  float* eps_row = p.eps + (size_t)n * p.ld;
-  const size_t obase = (size_t)n * p.k;
   const bool overflow = (u64)cand_count > (u64)p.capA;
   const u32 ncand = overflow ? (u32)p.capA : cand_count;
   const u32 novr = p.use_marks ? k : 0u;
@@ -904,79 +1085,33 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
   const int64_t su0 = (int64_t)rk * nw * seg_units < U ? (int64_t)rk * nw * seg_units : U;
   const int64_t su1 = (int64_t)(rk + 1) * nw * seg_units < U ? (int64_t)(rk + 1) * nw * seg_units : U;
 
-  for (int i = tid; i < kBins; i += blockDim.x) sh.hist[i] = 0;
-  for (u32 i = first_t; i < (u32)kSampleBins; i += stride_t) p.shist[(size_t)n * kSampleBins + i] = 0;
-  __syncthreads();
-  // ---- one sweep over the lists, a single wave of coalesced loads per step:
-  //   (a) the mask buffer of this round still holds the mask of two rounds ago: clear those words;
-  //   (b) the override scores (written by k_sample_cutoff's override clusters) that reach the
-  //       cutoff become composites and enter the histogram;
-  //   (c) the candidates (k_stream already dropped those on the previous support) enter it too ----
-  {
-    const u32 span = !dense && ncand > k ? ncand : k;
-    constexpr int kP0 = 8;  // items per thread in flight
-    for (u32 i0 = first_t; i0 < span; i0 += kP0 * stride_t) {
-      int32_t stale[kP0], j[kP0];
-      u32 key[kP0];
-      u64 c[kP0];
-#pragma unroll
-      for (int q = 0; q < kP0; ++q) {
-        const u32 i = i0 + q * stride_t;
-        const bool in_k = i < k;
-        stale[q] = (in_k && p.has_stale) ? p.cur_idx[obase + i] : -1;
-        j[q] = (in_k && p.use_marks) ? prev_idx[i] : -1;
-        key[q] = (in_k && p.use_marks) ? okey[i] : 0u;
-        c[q] = (!dense && i < ncand) ? A[i] : 0ull;
-      }
-#pragma unroll
-      for (int q = 0; q < kP0; ++q) {
-        const u32 i = i0 + q * stride_t;
-        if (stale[q] >= 0) mask[(u32)stale[q] >> 5] = 0u;
-        if (j[q] >= 0) {
-          const u64 oc = key[q] >= cutoff ? make_composite(key[q], (u32)j[q]) : 0ull;
-          O[i] = oc;
-          if (!dense && oc) atomicAdd(&sh.hist[select_bin(key[q], cutoff, bshift)], 1u);
-        }
-        if (c[q]) atomicAdd(&sh.hist[select_bin((u32)(c[q] >> 32), cutoff, bshift)], 1u);
-      }
-    }
-  }
-  __syncthreads();
-  if (!dense) flush_hist(sh.hist, ghist, kBins);
-  cl.sync();  // (1) cluster histogram complete; stale mask words cleared; override keys written
-
   u32 b1 = kFull, above1 = 0, nvalid = 0;
   bool took_dense = false;
-  if (!dense) {
-    load_and_find(sh, ghist, k, &b1, &above1, &nvalid);
-    if (b1 == kFull || overflow) dense = true;  // cutoff guessed too high, or the list overflowed
-    if (rk == 0 && tid == 0) ctl->n_valid = nvalid;
+  if (p.wide) {
+    // the sweep, the threshold and the classification were done by k_wide_hist and k_wide_classify
+    b1 = ctl->b1;
+    above1 = ctl->above1;
+    dense = ctl->go_dense != 0;
+  } else {
+    for (int i = tid; i < kBins; i += blockDim.x) sh.hist[i] = 0;
+    for (u32 i = first_t; i < (u32)kSampleBins; i += stride_t) p.shist[(size_t)n * kSampleBins + i] = 0;
+    __syncthreads();
+    post_sweep(p, n, first_t, stride_t, dense, ncand, cutoff, bshift, sh.hist);
+    __syncthreads();
+    if (!dense) flush_hist(sh.hist, ghist, kBins);
+    cl.sync();  // (1) cluster histogram complete; stale mask words cleared; override keys written
+    if (!dense) {
+      load_and_find(sh, ghist, k, &b1, &above1, &nvalid);
+      if (b1 == kFull || overflow) dense = true;  // cutoff guessed too high, or the list overflowed
+      if (rk == 0 && tid == 0) ctl->n_valid = nvalid;
+    }
+    if (!dense) {
+      post_classify(p, n, first_t, stride_t, ncand, novr, cutoff, bshift, b1);
+      cl.sync();  // (2) refinement list complete
+    }
   }
 
   if (!dense) {
-    // ---- classify: above the bin -> winner; inside it -> refinement list ----
-    // (candidates and overrides as one item list, eight loads per thread in flight)
-    {
-      const u32 total_items = ncand + novr;
-      const u32 iters = (total_items + 8 * stride_t - 1) / (8 * stride_t);
-      for (u32 it = 0; it < iters; ++it) {
-        u64 c[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          const u32 t = (it * 8 + q) * stride_t + first_t;
-          c[q] = t < ncand ? __ldcg(A + t) : (t < total_items ? __ldcg(O + (t - ncand)) : 0ull);
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          const u32 bin = c[q] ? select_bin((u32)(c[q] >> 32), cutoff, bshift) : 0u;
-          if (c[q] && bin > b1) set_winner(mask, composite_idx(c[q]));
-          const bool inbin = c[q] && bin == b1;
-          const u32 pos = warp_reserve_global(inbin, &ctl->bcount);
-          if (inbin) B[pos] = c[q];
-        }
-      }
-    }
-    cl.sync();  // (2) refinement list complete
     const u32 nB = __ldcg(&ctl->bcount);
     const u32 need = k - above1;
     if (nB <= blockDim.x) {
@@ -1057,6 +1192,10 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
       for (u32 i = first_t; i < k; i += stride_t) set_winner(mask, composite_idx(__ldcg(&A[i])));
     cl.sync();  // every winner bit is set
   }
+  if (p.wide) {  // k_wide_prefix and k_wide_emit take over
+    if (rk == 0 && tid == 0) ctl->took_dense = took_dense ? 1u : 0u;
+    return;
+  }
 
   // ---- emission.  The rank of a winner (its place in the ascending output) is the number of mask
   //      bits before it.  (E1) every warp of the cluster owns a fixed segment of the mask row and
@@ -1067,38 +1206,7 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
   //      threads, so a region dense with winners costs no more than a sparse one. ----
   __syncthreads();
   const int lane = tid & 31, warp = tid >> 5;
-  const u32 gw = rk * (u32)nw + (u32)warp;  // this warp's segment
-  const uint4* quads = reinterpret_cast<const uint4*>(mask);
-  u32* qpre = p.qprefix + (size_t)n * (p.W >> 2);
-  {
-    const int64_t wu0 = (int64_t)gw * seg_units < U ? (int64_t)gw * seg_units : U;
-    const int64_t wu1 = wu0 + seg_units < U ? wu0 + seg_units : U;
-    u32 running = 0;
-    for (int64_t ub = wu0; ub < wu1; ub += 128) {  // four rows of 32 units per step
-      uint4 x[4], y[4];
-#pragma unroll
-      for (int it = 0; it < 4; ++it) {
-        const int64_t u = ub + it * 32 + lane;
-        x[it] = u < wu1 ? __ldcg(quads + 2 * u) : make_uint4(0, 0, 0, 0);
-        y[it] = u < wu1 ? __ldcg(quads + 2 * u + 1) : make_uint4(0, 0, 0, 0);
-      }
-#pragma unroll
-      for (int it = 0; it < 4; ++it) {
-        const u32 cx = popc4(x[it]), c = cx + popc4(y[it]);
-        u32 inc = c;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const u32 t = __shfl_up_sync(kFull, inc, o);
-          if (lane >= o) inc += t;
-        }
-        const int64_t u = ub + it * 32 + lane;
-        const u32 pre = running + inc - c;
-        if (u < wu1) *reinterpret_cast<uint2*>(qpre + 2 * u) = make_uint2(pre, pre + cx);
-        running += __shfl_sync(kFull, inc, 31);
-      }
-    }
-    if (lane == 0) p.segtot[(size_t)n * kMaxSegments + gw] = running;
-  }
+  post_prefix_segment(p, n, rk * (u32)nw + (u32)warp, seg_units, lane);
   cl.sync();  // (3) segment totals and quad prefixes of the whole row are written
   u32* s_segbase = sh.spare;  // kMaxSegments <= kBins entries
   {
@@ -1115,60 +1223,93 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
       return;
     }
   }
-  {
-    // normal path: candidates and overrides as one item list; dense path: its k winners, nothing
-    // else.  Items below the threshold bin cannot have won and are skipped without touching memory.
-    const u32 nA = took_dense ? k : ncand;
-    const u32 total_items = nA + (took_dense ? 0u : novr);
-    for (u32 t0 = first_t; t0 < total_items; t0 += 4 * stride_t) {
-      u64 c[4];
-      uint4 qw[4];
-      u32 qp[4];
-      float vv[4];
-      bool live[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const u32 t = t0 + q * stride_t;
-        c[q] = t < nA ? __ldcg(A + t) : (t < total_items ? __ldcg(O + (t - nA)) : 0ull);
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const u32 idx = composite_idx(c[q]);
-        live[q] = c[q] != 0ull && (took_dense || select_bin((u32)(c[q] >> 32), cutoff, bshift) >= b1);
-        qw[q] = live[q] ? __ldcg(quads + (idx >> 7)) : make_uint4(0, 0, 0, 0);
-        qp[q] = live[q] ? __ldcg(qpre + (idx >> 7)) : 0u;
-        vv[q] = live[q] ? eps_row[idx] : 0.0f;
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        if (!live[q]) continue;
-        const u32 idx = composite_idx(c[q]);
-        const u32 w[4] = {qw[q].x, qw[q].y, qw[q].z, qw[q].w};
-        const u32 wsel = (idx >> 5) & 3u;
-        u32 before = 0, word = 0;
-#pragma unroll
-        for (int wi = 0; wi < 4; ++wi) {
-          if ((u32)wi < wsel) before += __popc(w[wi]);
-          if ((u32)wi == wsel) word = w[wi];
-        }
-        const u32 bm = 1u << (idx & 31);
-        if (word & bm) {
-          const u32 r = s_segbase[(idx >> 8) / (u32)seg_units] + qp[q] + before + __popc(word & (bm - 1u));
-          eps_row[idx] = 0.0f;  // a - a
-          if (p.pair_mode) {
-            // many pairs: one 8-byte store at the (random) rank instead of four 4-byte ones; k_unzip
-            // spreads the pairs over the four output arrays with sequential accesses afterwards
-            reinterpret_cast<uint2*>(B)[r] = make_uint2(idx, __float_as_uint(vv[q]));
-          } else {
-            p.out_idx[obase + r] = (int32_t)idx;
-            p.out_val[obase + r] = vv[q];
-            p.cur_idx[obase + r] = (int32_t)idx;
-            p.cur_val[obase + r] = vv[q];
-          }
-        }
-      }
-    }
+  post_emit(p, n, first_t, stride_t, ncand, novr, took_dense, cutoff, bshift, b1, s_segbase, seg_units);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Wide mode (N*k large): the list phases of k_post as kernels of their own on the whole grid, blockIdx.y
+// = worker, because there the lists are long enough for throughput, not latency, to decide:
+//   k_wide_hist -> k_wide_classify -> k_post (refinement or dense path only) -> k_wide_prefix -> k_wide_emit.
+// The mask row is cut into kMaxSegments segments whatever the grid.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_wide_hist(PostArgs p) {
+  __shared__ u32 s_hist[kBins];
+  grid_dependency_begin();
+  const int n = blockIdx.y, tid = threadIdx.x;
+  const u32 stride_t = gridDim.x * blockDim.x, first_t = blockIdx.x * blockDim.x + tid;
+  const WorkerCtl* ctl = p.ctl + n;
+  const u32 cutoff = ctl->cutoff, bshift = ctl->bin_shift, cand_count = ctl->cand_count;
+  const bool dense = ctl->force_dense != 0;
+  const u32 ncand = (u64)cand_count > (u64)p.capA ? (u32)p.capA : cand_count;
+  for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
+  for (u32 i = first_t; i < (u32)kSampleBins; i += stride_t) p.shist[(size_t)n * kSampleBins + i] = 0;
+  __syncthreads();
+  post_sweep(p, n, first_t, stride_t, dense, ncand, cutoff, bshift, s_hist);
+  __syncthreads();
+  if (!dense) flush_hist(s_hist, p.ghist + (size_t)n * 4 * kBins, kBins);
+}
+
+__global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_wide_classify(PostArgs p) {
+  __shared__ __align__(16) PostShared sh;
+  grid_dependency_begin();
+  const int n = blockIdx.y, tid = threadIdx.x;
+  const u32 stride_t = gridDim.x * blockDim.x, first_t = blockIdx.x * blockDim.x + tid;
+  WorkerCtl* ctl = p.ctl + n;
+  const u32 cutoff = ctl->cutoff, bshift = ctl->bin_shift, cand_count = ctl->cand_count;
+  bool dense = ctl->force_dense != 0;
+  const bool overflow = (u64)cand_count > (u64)p.capA;
+  const u32 ncand = overflow ? (u32)p.capA : cand_count;
+  u32 b1 = kFull, above1 = 0, nvalid = 0;
+  if (!dense) {  // every block finds the threshold bin by itself (all get the same answer)
+    load_and_find(sh, p.ghist + (size_t)n * 4 * kBins, (u32)p.k, &b1, &above1, &nvalid);
+    if (b1 == kFull || overflow) dense = true;
   }
+  if (blockIdx.x == 0 && tid == 0) {
+    ctl->b1 = b1;
+    ctl->above1 = above1;
+    ctl->go_dense = dense ? 1u : 0u;
+    ctl->n_valid = nvalid;
+  }
+  if (!dense) post_classify(p, n, first_t, stride_t, ncand, p.use_marks ? (u32)p.k : 0u, cutoff, bshift, b1);
+}
+
+__global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_wide_prefix(PostArgs p) {
+  grid_dependency_begin();
+  const int n = blockIdx.y;
+  const int lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  const int64_t U = p.W >> 3;
+  const int64_t seg_units = (U + kMaxSegments - 1) / kMaxSegments;
+  for (u32 seg = blockIdx.x * nw + (threadIdx.x >> 5); seg < (u32)kMaxSegments; seg += gridDim.x * nw)
+    post_prefix_segment(p, n, seg, seg_units, lane);
+}
+
+__global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_wide_emit(PostArgs p) {
+  __shared__ u32 s_segbase[kMaxSegments];
+  __shared__ u32 s_scan[33];
+  grid_dependency_begin();
+  const int n = blockIdx.y, tid = threadIdx.x;
+  const u32 stride_t = gridDim.x * blockDim.x, first_t = blockIdx.x * blockDim.x + tid;
+  const WorkerCtl* ctl = p.ctl + n;
+  const u32 cutoff = ctl->cutoff, bshift = ctl->bin_shift, cand_count = ctl->cand_count;
+  const u32 b1 = ctl->b1;
+  const bool took_dense = ctl->took_dense != 0;
+  const u32 ncand = (u64)cand_count > (u64)p.capA ? (u32)p.capA : cand_count;
+  const int64_t U = p.W >> 3;
+  const int64_t seg_units = (U + kMaxSegments - 1) / kMaxSegments;
+  u32 total;
+  const u32 t = tid < kMaxSegments ? __ldcg(&p.segtot[(size_t)n * kMaxSegments + tid]) : 0u;
+  const u32 base = block_excl_scan(t, s_scan, &total);  // blockDim.x >= kMaxSegments
+  if (tid < kMaxSegments) {
+    s_segbase[tid] = base;
+    if (blockIdx.x == 0) p.segbase[(size_t)n * kMaxSegments + tid] = base;  // for k_aggregate
+  }
+  __syncthreads();
+  if (total != (u32)p.k) {
+    if (blockIdx.x == 0 && tid == 0) atomicOr(&p.gctl->err, kErrCountMismatch);
+    return;
+  }
+  post_emit(p, n, first_t, stride_t, ncand, p.use_marks ? (u32)p.k : 0u, took_dense, cutoff, bshift, b1, s_segbase,
+            seg_units);
 }
 
 // After k_post in pair mode: (index, value) pairs, in rank order in the workers' B lists, go to the
@@ -1428,6 +1569,10 @@ Layout make_layout(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
 }
 
 constexpr int kMaxProfile = 4096;
+#ifndef REGTOPK_MANY_PAIRS
+#define REGTOPK_MANY_PAIRS 262144
+#endif
+constexpr int64_t kManyPairs = REGTOPK_MANY_PAIRS;  // N*k from which the list phases run in wide mode
 
 }  // namespace
 
@@ -1445,6 +1590,7 @@ struct regtopk_ctx {
   int sticky;        // first CUDA error seen
   int num_sms;
   int cluster;       // blocks per worker in k_post
+  int many_pairs;    // N*k is large (or the testing flag is set): wide kernels and pair-mode emission
   int stream_blocks[5];
   int64_t launches;
   int profiling;
@@ -1605,6 +1751,7 @@ int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const reg
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->num_sms = sms > 0 ? sms : 148;
   c->cluster = choose_cluster(N);
+  c->many_pairs = (k * (int64_t)N >= kManyPairs || (params->flags & REGTOPK_FLAG_FORCE_WIDE_LISTS)) ? 1 : 0;
   float* om = static_cast<float*>(malloc(sizeof(float) * N));
   if (!om) { free(c); return REGTOPK_ERR_INVALID_ARG; }
   for (int n = 0; n < N; ++n) om[n] = params->omega ? params->omega[n] : 1.0f / (float)N;
@@ -1695,7 +1842,23 @@ int step_impl(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_i
   pa.out_idx = out_idx; pa.out_val = out_val;
   pa.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); pa.cur_val = at<float>(c, L.off_val[c->cur]);
   pa.use_marks = use_marks; pa.has_stale = c->round >= 2;
-  pa.pair_mode = c->k * (int64_t)c->N >= 262144;
+  pa.pair_mode = c->many_pairs;
+  pa.wide = c->many_pairs;
+  // wide kernels: the grid's blocks split evenly over the workers (blockIdx.y = worker)
+  cudaLaunchConfig_t wcfg;
+  cudaLaunchAttribute wattr[2];
+  {
+    int bx = c->num_sms / c->N;
+    if (bx < 1) bx = 1;
+    launch_config(&wcfg, wattr, (unsigned)bx, 1, kBlockPost, 0, c->stream);
+    wcfg.gridDim = dim3((unsigned)bx, (unsigned)c->N, 1);
+  }
+  if (pa.wide) {
+    cudaLaunchKernelEx(&wcfg, k_wide_hist, pa);
+    if ((rc = after_launch(c))) return rc;
+    cudaLaunchKernelEx(&wcfg, k_wide_classify, pa);
+    if ((rc = after_launch(c))) return rc;
+  }
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[2];
   post_config(&cfg, attr, c->N, c->cluster, kBlockPost, c->stream);
@@ -1703,6 +1866,12 @@ int step_impl(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_i
   c->launches++;
   if (le != cudaSuccess) return note_cuda(c, le);
   if ((rc = note_cuda(c, cudaGetLastError()))) return rc;
+  if (pa.wide) {
+    cudaLaunchKernelEx(&wcfg, k_wide_prefix, pa);
+    if ((rc = after_launch(c))) return rc;
+    cudaLaunchKernelEx(&wcfg, k_wide_emit, pa);
+    if ((rc = after_launch(c))) return rc;
+  }
   if (pa.pair_mode) {
     UnzipArgs ua;
     ua.candB = pa.candB; ua.stride = L.stride; ua.k = c->k; ua.N = c->N;
@@ -1754,7 +1923,10 @@ int regtopk_aggregate_update(regtopk_ctx* c, float* theta, float eta, float* out
   a.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); a.cur_val = at<float>(c, L.off_val[c->cur]);
   a.prev_idx = at<int32_t>(c, L.off_idx[c->cur ^ 1]);
   a.bitmask = at<u32>(c, L.off_mask[c->cur]); a.qprefix = at<u32>(c, L.off_qprefix); a.segbase = at<u32>(c, L.off_segbase);
-  a.seg_units = ((L.W >> 3) + (int64_t)c->cluster * (kBlockPost / 32) - 1) / ((int64_t)c->cluster * (kBlockPost / 32));
+  {  // segments of the mask row as the emission cut them: one per warp of the k_post cluster, kMaxSegments in wide mode
+    const int64_t nseg = c->many_pairs ? kMaxSegments : (int64_t)c->cluster * (kBlockPost / 32);
+    a.seg_units = ((L.W >> 3) + nseg - 1) / nseg;
+  }
   a.W = L.W;
   a.omega = at<float>(c, L.off_omega);
   a.has_prev = c->round >= 1;

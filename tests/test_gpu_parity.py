@@ -188,6 +188,41 @@ def test_sample_underestimates_cutoff():
     run_parity(rounds, d, N, k, 4.0, expect_dense=True)
 
 
+# ---- the list handling of large N*k (separate full-grid kernels, pairs unzipped afterwards), forced at small
+#      sizes ------------------------------------------------------------------------------------------------
+WIDE = binding.FLAG_FORCE_WIDE_LISTS
+
+
+@pytest.mark.parametrize("d,N,k", [(1, 1, 1), (7, 3, 7), (33, 2, 5), (512, 1, 512), (513, 3, 1), (4096, 8, 41),
+                                   (65537, 2, 655), (200003, 4, 2000), (200003, 2, 200003), (1_000_003, 2, 10_000),
+                                   (3001, 33, 7), (70_000, 150, 70)])
+@pytest.mark.parametrize("mu", [4.0, 0.0])
+def test_wide_lists_sizes(d, N, k, mu):
+    run_parity(gauss_rounds(N, d, 4, seed=d + N + 1), d, N, k, mu, flags=WIDE)
+
+
+def test_wide_lists_dense_path_ties_bf16_exponent_inplace():
+    run_parity(gauss_rounds(3, 90_001, 4, seed=21), 90_001, 3, 900, 4.0, flags=WIDE | binding.FLAG_FORCE_DENSE_SELECT,
+               expect_dense=True)
+    run_parity(gauss_rounds(3, 150_000, 4, seed=8, quant=2), 150_000, 3, 1500, 4.0, flags=WIDE)
+    run_parity(gauss_rounds(2, 100_001, 4, seed=10, ld=100_008, dtype=torch.bfloat16), 100_001, 2, 1000, 4.0, flags=WIDE)
+    run_parity(gauss_rounds(3, 80_000, 4, seed=51), 80_000, 3, 800, 2.0, y=0.5, flags=WIDE, inplace=lambda t: t % 2 == 0)
+
+
+def test_wide_lists_sample_misses_and_long_run():
+    d, N, k = 1_000_000, 2, 5000
+    pos = torch.from_numpy(_sample_positions(d))
+    rounds = []
+    for x in gauss_rounds(N, d, 3, seed=30):
+        x[:, pos] *= 100.0
+        rounds.append(x)
+    run_parity(rounds, d, N, k, 4.0, expect_dense=True, flags=WIDE)
+    w = synth.workload("resnet18", scale_to=400_000)
+    s = synth.GradientStream(w, device="cpu", seed=31, pad_to=8)
+    st = run_parity((s.next() for _ in range(20)), w.d, w.N, w.k_values()[1], w.mu, threads=8, flags=WIDE)
+    assert st["dense_select_workers"] == 0, st
+
+
 # ---- accumulate-in-place calls: the caller adds g into the library's rows, the library only scans them ------
 @pytest.mark.parametrize("d,N,k", [(1, 1, 1), (7, 3, 7), (513, 3, 1), (4096, 8, 41), (65537, 2, 655),
                                    (200003, 4, 2000), (200003, 2, 200003), (1_000_003, 2, 1000), (70_000, 150, 70)])
