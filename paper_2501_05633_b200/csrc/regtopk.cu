@@ -20,6 +20,11 @@
 //   k_aggregate       server sum in worker order, one thread per sent pair, ranks looked up through
 //                     the prefix counts written during emission
 //
+// When N*k is large the list phases of k_post run as kernels of their own on the whole grid instead
+// (k_wide_hist, k_wide_classify, k_post for the refinement only, k_wide_prefix, k_wide_emit, k_unzip): see
+// "Wide mode" below.  regtopk_worker_step_inplace uses a read-only variant of k_stream on rows into which
+// the caller has already added the gradients.
+//
 // The selection key of an entry is the bit pattern of its non-negative binary32 score, which orders
 // like the score; the 64-bit composite (key << 32 | ~index) orders like (score descending, index
 // ascending) and is unique per entry, so "the k largest composites" is the mask with the
