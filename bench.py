@@ -24,7 +24,7 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_stream launch from the ncu capture summarised in
 # profiles/k_stream_resnet18_fp32_full.md; valid for that workload and the kernel as captured.
-NCU_STREAM_TRAFFIC = {"resnet18": 1026.1e6}
+NCU_STREAM_TRAFFIC = {"resnet18": 1027.1e6}
 
 METRIC = "RegTop-k step throughput (G coords/s, all N workers) and achieved HBM GB/s vs peak"
 UNIT = "G coords/s"
