@@ -618,9 +618,16 @@ __global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC, INPLACE
   const char* grow = nullptr;
   const u32* marks = nullptr;
 
-  for (int64_t c = (int64_t)blockIdx.x * (kStreamThreads / 32) + warp; c < total; c += nwarps) {
-    const int n = (int)(c / chunks_per_row);
-    const int64_t base = (c - (int64_t)n * chunks_per_row) * S::kChunk;
+  // row and position of the warp's chunk advance incrementally: one 64-bit division up front, none per chunk
+  const int64_t cfirst = (int64_t)blockIdx.x * (kStreamThreads / 32) + warp;
+  int64_t row = cfirst / chunks_per_row, in_row = cfirst - row * chunks_per_row;
+  const int64_t step_rows = nwarps / chunks_per_row, step_in = nwarps - step_rows * chunks_per_row;
+  for (int64_t c = cfirst; c < total; c += nwarps) {
+    const int n = (int)row;
+    const int64_t base = in_row * S::kChunk;
+    row += step_rows;
+    in_row += step_in;
+    if (in_row >= chunks_per_row) { in_row -= chunks_per_row; ++row; }
     if (n != cur_n) {
       if (cur_n >= 0) stream_flush(list, wcount, p.ctl + cur_n, p.cand + (size_t)cur_n * p.stride, p.cap, marks, lane);
       cur_n = n;
