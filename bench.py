@@ -283,6 +283,18 @@ def main():
             a1.record()
         torch.cuda.synchronize()
         lib_only_ms = sum(a0.elapsed_time(a1) for a0, a1 in evs) / nlib
+    # ---- round 0 (no previous support: Algorithm 1) on its own ----
+    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    round0 = []
+    for _ in range(3):
+        lib.state_reset()
+        torch.cuda.synchronize()
+        r0.record()
+        step(0)
+        r1.record()
+        torch.cuda.synchronize()
+        round0.append(r0.elapsed_time(r1))
+    round0_ms = statistics.median(round0)
     # ---- end to end through host buffers ----
     e2e_s = float("nan")
     if args.e2e_steps > 0 and not inplace:
@@ -322,7 +334,8 @@ def main():
                        "step_frac_of_8TBs": step_gbs / 8000.0,
                        "dense_select_workers": stats_end["dense_select_workers"],
                        "candidates_last": stats_end["candidates_last"],
-                       "ms_per_step_with_kernel_events": ms_prof / nprof},
+                       "ms_per_step_with_kernel_events": ms_prof / nprof,
+                       "round0_ms": round0_ms},
             "clocks": clocks,
             "e2e": {"value": (world * coords * args.e2e_steps / e2e_all / 1e9) if (args.e2e_steps > 0 and not inplace) else None, "unit": UNIT,
                     "h2d_bytes_per_step": w.N * stream.ld * bpe, "d2h_bytes_per_step": 2 * w.N * k * 4 + w.d * 4},
