@@ -1376,14 +1376,16 @@ struct AggArgs {
 };
 
 __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
-  const int64_t npairs = p.k * p.N;
-  const int64_t total = p.has_prev ? 2 * npairs : npairs;
+  // grid: x over the pairs of one worker, y = worker, z = 0 for this round's pairs, 1 for the previous round's
   const int64_t Q = p.W >> 2;
+  const int n = blockIdx.y;
+  const bool prev_pass = blockIdx.z != 0;
+  const u32 seg_units = (u32)p.seg_units;
   grid_dependency_begin();
-  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
-       t += (int64_t)gridDim.x * blockDim.x) {
-    if (t >= npairs) {  // a pair of the previous round
-      const int32_t j = p.prev_idx[t - npairs];
+  for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < p.k; r += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t t = (int64_t)n * p.k + r;
+    if (prev_pass) {  // a pair of the previous round
+      const int32_t j = p.prev_idx[t];
       const size_t wi = (size_t)(j >> 5);
       const u32 bm = 1u << (j & 31);
       u32 any = 0;
@@ -1397,13 +1399,12 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
       if (!(any & bm)) p.g[j] = 0.0f;
       continue;
     }
-    const int n = (int)(t / p.k);
     const int32_t j = p.cur_idx[t];
     const size_t wi = (size_t)(j >> 5);
     const size_t qi = wi >> 2;
     const int wsub = (int)(wi & 3);
     const u32 bm = 1u << (j & 31);
-    const size_t seg = (size_t)((int64_t)(wi >> 3) / p.seg_units);
+    const size_t seg = (size_t)((u32)(wi >> 3) / seg_units);
     // a higher-numbered worker that sent j owns it
     bool owned = true;
     for (int m0 = n + 1; m0 < p.N && owned; m0 += 8) {
@@ -1943,13 +1944,15 @@ int regtopk_aggregate_update(regtopk_ctx* c, float* theta, float eta, float* out
   a.omega = at<float>(c, L.off_omega);
   a.has_prev = c->round >= 1;
   a.theta = theta; a.eta = eta;
-  const int64_t threads = (a.has_prev ? 2 : 1) * c->k * (int64_t)c->N;
-  int64_t blocks = (threads + 255) / 256;
-  if (blocks > (int64_t)c->num_sms * 32) blocks = (int64_t)c->num_sms * 32;
   {
+    const int passes = a.has_prev ? 2 : 1;
+    int64_t bx = (c->k + 255) / 256;
+    const int64_t cap_x = ((int64_t)c->num_sms * 32 + (int64_t)c->N * passes - 1) / ((int64_t)c->N * passes);
+    if (bx > cap_x) bx = cap_x;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[2];
-    launch_config(&cfg, attr, (unsigned)blocks, 1, 256, 0, c->stream);
+    launch_config(&cfg, attr, (unsigned)bx, 1, 256, 0, c->stream);
+    cfg.gridDim = dim3((unsigned)bx, (unsigned)c->N, (unsigned)passes);
     cudaLaunchKernelEx(&cfg, k_aggregate, a);
   }
   int rc = after_launch(c);
