@@ -482,6 +482,14 @@ def test_full_size_workloads(name, ki, rounds):
                expect_dense=False)
 
 
+def test_full_size_inplace_calls():
+    """The accumulate-in-place calls at the benchmark's size and layout (ResNet-18 shape, k = 0.1 %)."""
+    w = synth.workload("resnet18")
+    s = synth.GradientStream(w, device="cuda", seed=0, pad_to=32)
+    run_parity((s.next() for _ in range(3)), w.d, w.N, w.k_values()[0], w.mu, select_mode=1, threads=8,
+               expect_dense=False, inplace=lambda t: True)
+
+
 # ---- full benchmark sizes too large to sort on the host: certified instead of compared --------------------------
 def _certified_round(lib, ora_api, w, k, grads, eps_before, prev, g_prev, omega):
     """One round of the library, checked against the oracle without a sort: the oracle's accumulator and
