@@ -158,7 +158,8 @@ typedef struct {
   int64_t dense_select_workers; /* worker-rounds that needed the dense exact path (sampled cutoff missed) */
   int64_t candidates_last;      /* candidates gathered in the last round, summed over workers             */
   int64_t candidate_capacity;   /* per-worker capacity of the candidate list                              */
-  int64_t device_error_bits;    /* 0, or which internal consistency check failed (1 count, 2 dense, 4 refine) */
+  int64_t device_error_bits;    /* 0, or which internal consistency check failed (1 count, 2 dense, 4 refine; 8: a
+                                   range check of the checked build, -DREGTOPK_DEBUG=1) */
 } regtopk_stats;
 
 /* Synchronises the stream and fills *out (host). */

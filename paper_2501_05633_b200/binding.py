@@ -59,6 +59,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return _LIB
 
 
+def build_checked(force: bool = False) -> str:
+    """The same library with -DREGTOPK_DEBUG=1 (every data-dependent index is range-checked on the device; a bad
+    one is counted and skipped, and status() then reports an internal error), as libregtopk_checked.so beside
+    the release library.  Used by tests/test_gpu_checked_build.py; nothing else loads it."""
+    out = os.path.join(_PKG, "libregtopk_checked.so")
+    if not force and os.path.exists(out) and os.path.getmtime(out) >= max(
+            os.path.getmtime(_SRC), os.path.getmtime(os.path.join(_INC, "regtopk.h"))):
+        return out
+    subprocess.run(["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+                    "-DREGTOPK_DEBUG=1", "-I", _INC, "--shared", "-Xcompiler", "-fPIC", "-o", out, _SRC], check=True)
+    return out
+
+
 _lib = None
 
 

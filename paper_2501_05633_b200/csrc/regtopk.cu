@@ -67,7 +67,21 @@ constexpr int kMaxCluster = 16;
 constexpr int kMaxSegments = kMaxCluster * 32;  // mask segments per row: one per warp of a k_post cluster
 constexpr u32 kFull = 0xFFFFFFFFu;
 
-enum : u32 { kErrCountMismatch = 1u, kErrDenseSelect = 2u, kErrRefine = 4u };
+enum : u32 { kErrCountMismatch = 1u, kErrDenseSelect = 2u, kErrRefine = 4u, kErrBounds = 8u };
+
+// Checked build (-DREGTOPK_DEBUG=1): every access whose index is computed from data (a candidate's
+// index, a rank, a list position) is tested against its array's extent first; an index out of range is
+// counted here and the access skipped, and regtopk_status then reports REGTOPK_ERR_INTERNAL.  Nothing
+// traps.  The release build compiles the tests away.
+#ifndef REGTOPK_DEBUG
+#define REGTOPK_DEBUG 0
+#endif
+#if REGTOPK_DEBUG
+__device__ unsigned int g_bounds_faults;
+#define RT_INB(cond) ((cond) ? true : (atomicAdd(&g_bounds_faults, 1u), false))
+#else
+#define RT_INB(cond) true
+#endif
 
 struct WorkerCtl {
   u32 cutoff;       // candidate cutoff key of this round
@@ -705,16 +719,16 @@ __global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC, INPLACE
           const u32 lt = (1u << lane) - 1u;
           u32 m;
           m = __ballot_sync(kFull, h0);
-          if (h0) list[wcount + __popc(m & lt)] = make_composite(k0, (u32)j);
+          if (h0 && RT_INB(wcount + __popc(m & lt) < (u32)kWarpList)) list[wcount + __popc(m & lt)] = make_composite(k0, (u32)j);
           wcount += __popc(m);
           m = __ballot_sync(kFull, h1);
-          if (h1) list[wcount + __popc(m & lt)] = make_composite(k1, (u32)j + 1);
+          if (h1 && RT_INB(wcount + __popc(m & lt) < (u32)kWarpList)) list[wcount + __popc(m & lt)] = make_composite(k1, (u32)j + 1);
           wcount += __popc(m);
           m = __ballot_sync(kFull, h2);
-          if (h2) list[wcount + __popc(m & lt)] = make_composite(k2, (u32)j + 2);
+          if (h2 && RT_INB(wcount + __popc(m & lt) < (u32)kWarpList)) list[wcount + __popc(m & lt)] = make_composite(k2, (u32)j + 2);
           wcount += __popc(m);
           m = __ballot_sync(kFull, h3);
-          if (h3) list[wcount + __popc(m & lt)] = make_composite(k3, (u32)j + 3);
+          if (h3 && RT_INB(wcount + __popc(m & lt) < (u32)kWarpList)) list[wcount + __popc(m & lt)] = make_composite(k3, (u32)j + 3);
           wcount += __popc(m);
           if (wcount >= kWarpList - 128)  // the next four elements per lane add at most 128
             stream_flush(list, wcount, p.ctl + cur_n, p.cand + (size_t)cur_n * p.stride, p.cap, marks, lane);
@@ -788,8 +802,8 @@ __device__ __forceinline__ u32 warp_reserve_global(bool pred, u32* counter) {
   return base + (u32)__popc(m & ((1u << lane) - 1u));
 }
 
-__device__ __forceinline__ void set_winner(u32* mask, u32 idx) {
-  atomicOr(&mask[idx >> 5], 1u << (idx & 31));
+__device__ __forceinline__ void set_winner(u32* mask, u32 idx, int64_t d) {
+  if (RT_INB((int64_t)idx < d)) atomicOr(&mask[idx >> 5], 1u << (idx & 31));
 }
 
 __device__ __forceinline__ u32 select_bin(u32 key, u32 cutoff, u32 shift) {
@@ -829,7 +843,7 @@ __device__ __forceinline__ u32 dense_key(const PostArgs& p, int n, int64_t j) {
 
 // One block: among list[0..count) (count <= blockDim.x, unique composites) set the `need` largest as
 // winners, but only those whose mask word lies in [w0, w1) (the caller's share of the mask).
-__device__ void refine_small(PostShared& sh, u32* mask, const u64* list, u32 count, u32 need,
+__device__ void refine_small(PostShared& sh, u32* mask, int64_t d, const u64* list, u32 count, u32 need,
                              int64_t w0, int64_t w1) {
   u64* s_items = reinterpret_cast<u64*>(sh.hist);
   const int tid = threadIdx.x;
@@ -845,7 +859,7 @@ __device__ void refine_small(PostShared& sh, u32* mask, const u64* list, u32 cou
     if (wi >= w0 && wi < w1) {
       u32 above = 0;
       for (u32 j = 0; j < count; ++j) above += s_items[j] > mine ? 1u : 0u;
-      if (above < need) set_winner(mask, idx);
+      if (above < need) set_winner(mask, idx, d);
     }
   }
   __syncthreads();
@@ -854,7 +868,7 @@ __device__ void refine_small(PostShared& sh, u32* mask, const u64* list, u32 cou
 // Leader block only: the `need` largest composites of list[0..count), any count (long runs of equal
 // keys end up here).  Eight histogram passes over the list fix the need-th largest composite byte by
 // byte, without moving the list; a last pass sets everything at or above it.
-__device__ void refine_large(PostShared& sh, u32* mask, GlobalCtl* gctl, const u64* list, u32 count,
+__device__ void refine_large(PostShared& sh, u32* mask, int64_t d, GlobalCtl* gctl, const u64* list, u32 count,
                              u32 need) {
   const int tid = threadIdx.x;
   if (need == 0) return;
@@ -879,7 +893,7 @@ __device__ void refine_large(PostShared& sh, u32* mask, GlobalCtl* gctl, const u
   }
   for (u32 i = tid; i < count; i += blockDim.x) {
     const u64 c = __ldcg(&list[i]);
-    if (c >= prefix) set_winner(mask, composite_idx(c));
+    if (c >= prefix) set_winner(mask, composite_idx(c), d);
   }
 }
 
@@ -923,7 +937,7 @@ __device__ __forceinline__ void post_sweep(const PostArgs& p, int n, u32 first_t
 #pragma unroll
     for (int q = 0; q < kP0; ++q) {
       const u32 i = i0 + q * stride_t;
-      if (stale[q] >= 0) mask[(u32)stale[q] >> 5] = 0u;
+      if (stale[q] >= 0 && RT_INB((int64_t)stale[q] < p.d)) mask[(u32)stale[q] >> 5] = 0u;
       if (j[q] >= 0) {
         const u64 oc = key[q] >= cutoff ? make_composite(key[q], (u32)j[q]) : 0ull;
         O[i] = oc;
@@ -955,10 +969,10 @@ __device__ __forceinline__ void post_classify(const PostArgs& p, int n, u32 firs
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
       const u32 bin = c[q] ? select_bin((u32)(c[q] >> 32), cutoff, bshift) : 0u;
-      if (c[q] && bin > b1) set_winner(mask, composite_idx(c[q]));
+      if (c[q] && bin > b1) set_winner(mask, composite_idx(c[q]), p.d);
       const bool inbin = c[q] && bin == b1;
       const u32 pos = warp_reserve_global(inbin, &ctl->bcount);
-      if (inbin) B[pos] = c[q];
+      if (inbin && RT_INB((int64_t)pos < p.stride)) B[pos] = c[q];
     }
   }
 }
@@ -1029,7 +1043,7 @@ __device__ __forceinline__ void post_emit(const PostArgs& p, int n, u32 first_t,
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const u32 idx = composite_idx(c[q]);
-      live[q] = c[q] != 0ull && (took_dense || select_bin((u32)(c[q] >> 32), cutoff, bshift) >= b1);
+      live[q] = c[q] != 0ull && (took_dense || select_bin((u32)(c[q] >> 32), cutoff, bshift) >= b1) && RT_INB((int64_t)idx < p.d);
       qw[q] = live[q] ? __ldcg(quads + (idx >> 7)) : make_uint4(0, 0, 0, 0);
       qp[q] = live[q] ? __ldcg(qpre + (idx >> 7)) : 0u;
       vv[q] = live[q] ? eps_row[idx] : 0.0f;
@@ -1047,8 +1061,9 @@ __device__ __forceinline__ void post_emit(const PostArgs& p, int n, u32 first_t,
         if ((u32)wi == wsel) word = w[wi];
       }
       const u32 bm = 1u << (idx & 31);
-      if (word & bm) {
+      if ((word & bm) && RT_INB((idx >> 8) / (u32)seg_units < (u32)kMaxSegments)) {
         const u32 r = s_segbase[(idx >> 8) / (u32)seg_units] + qp[q] + before + __popc(word & (bm - 1u));
+        if (!RT_INB(r < k)) continue;
         eps_row[idx] = 0.0f;  // a - a
         if (p.pair_mode) {
           // many pairs: one 8-byte store at the (random) rank instead of four 4-byte ones; k_unzip
@@ -1128,9 +1143,9 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
     const u32 need = k - above1;
     if (nB <= blockDim.x) {
       // every block ranks the short list itself and sets the winners of its own share of the mask
-      refine_small(sh, mask, B, nB, need, su0 * 8, su1 * 8);
+      refine_small(sh, mask, p.d, B, nB, need, su0 * 8, su1 * 8);
     } else {
-      if (rk == 0) refine_large(sh, mask, p.gctl, B, nB, need);
+      if (rk == 0) refine_large(sh, mask, p.d, p.gctl, B, nB, need);
       cl.sync();  // (2b) the leader's winners are set
     }
   } else {
@@ -1195,13 +1210,13 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
       const bool tie = j < c1 && dense_key(p, n, j) == T;
       u32 total;
       const u32 rank = taken + block_excl_scan(tie ? 1u : 0u, sh.scan, &total);
-      if (tie && rank < need) A[n_gt + rank] = make_composite(T, (u32)j);
+      if (tie && rank < need && RT_INB(n_gt + rank < k)) A[n_gt + rank] = make_composite(T, (u32)j);
       taken += total;
     }
     cl.sync();  // winner list complete
     if (rk == 0 && tid == 0 && (bad || __ldcg(&ctl->acount) != n_gt)) atomicOr(&p.gctl->err, kErrDenseSelect);
     if (!bad)
-      for (u32 i = first_t; i < k; i += stride_t) set_winner(mask, composite_idx(__ldcg(&A[i])));
+      for (u32 i = first_t; i < k; i += stride_t) set_winner(mask, composite_idx(__ldcg(&A[i])), p.d);
     cl.sync();  // every winner bit is set
   }
   if (p.wide) {  // k_wide_prefix and k_wide_emit take over
@@ -1359,6 +1374,7 @@ __global__ void __launch_bounds__(256) k_unzip(UnzipArgs p) {
 // ---------------------------------------------------------------------------------------------
 struct AggArgs {
   float* g;
+  int64_t d;
   int N;
   int64_t k;
   const int32_t* cur_idx;
@@ -1386,6 +1402,7 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
     const int64_t t = (int64_t)n * p.k + r;
     if (prev_pass) {  // a pair of the previous round
       const int32_t j = p.prev_idx[t];
+      if (!RT_INB(j >= 0 && (int64_t)j < p.d)) continue;
       const size_t wi = (size_t)(j >> 5);
       const u32 bm = 1u << (j & 31);
       u32 any = 0;
@@ -1400,11 +1417,13 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
       continue;
     }
     const int32_t j = p.cur_idx[t];
+    if (!RT_INB(j >= 0 && (int64_t)j < p.d)) continue;
     const size_t wi = (size_t)(j >> 5);
     const size_t qi = wi >> 2;
     const int wsub = (int)(wi & 3);
     const u32 bm = 1u << (j & 31);
     const size_t seg = (size_t)((u32)(wi >> 3) / seg_units);
+    if (!RT_INB(seg < (size_t)kMaxSegments)) continue;
     // a higher-numbered worker that sent j owns it
     bool owned = true;
     for (int m0 = n + 1; m0 < p.N && owned; m0 += 8) {
@@ -1439,6 +1458,7 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
         }
         has[u] = (mine & bm) != 0u;
         rank += __popc(mine & (bm - 1u));
+        if (has[u] && !RT_INB((int64_t)rank < p.k)) has[u] = false;
         v[u] = has[u] ? p.cur_val[(size_t)(m0 + u) * p.k + rank] : 0.0f;
       }
 #pragma unroll
@@ -1932,7 +1952,7 @@ int regtopk_aggregate_update(regtopk_ctx* c, float* theta, float eta, float* out
   if (!c->stepped) return REGTOPK_ERR_SEQUENCE;
   const Layout& L = c->L;
   AggArgs a;
-  a.g = at<float>(c, L.off_g); a.N = c->N; a.k = c->k;
+  a.g = at<float>(c, L.off_g); a.d = c->d; a.N = c->N; a.k = c->k;
   a.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); a.cur_val = at<float>(c, L.off_val[c->cur]);
   a.prev_idx = at<int32_t>(c, L.off_idx[c->cur ^ 1]);
   a.bitmask = at<u32>(c, L.off_mask[c->cur]); a.qprefix = at<u32>(c, L.off_qprefix); a.segbase = at<u32>(c, L.off_segbase);
@@ -2066,6 +2086,11 @@ int regtopk_status(regtopk_ctx* c) {
   if (!rc) rc = note_cuda(c, cudaStreamSynchronize(c->stream));
   if (c->sticky) return c->sticky;
   if (rc) return rc;
+#if REGTOPK_DEBUG
+  unsigned int faults = 0;
+  if (cudaMemcpyFromSymbol(&faults, g_bounds_faults, sizeof faults) != cudaSuccess) return note_cuda(c, cudaErrorUnknown);
+  if (faults) return REGTOPK_ERR_INTERNAL;
+#endif
   return h.err ? REGTOPK_ERR_INTERNAL : REGTOPK_OK;
 }
 
@@ -2086,6 +2111,11 @@ int regtopk_get_stats(regtopk_ctx* c, regtopk_stats* out) {
     for (int n = 0; n < c->N; ++n) out->candidates_last += w[n].cand_count;
     out->candidate_capacity = c->L.capA;
     out->device_error_bits = (int64_t)h.err;
+#if REGTOPK_DEBUG
+    unsigned int faults = 0;
+    if (cudaMemcpyFromSymbol(&faults, g_bounds_faults, sizeof faults) == cudaSuccess && faults)
+      out->device_error_bits |= (int64_t)kErrBounds;
+#endif
   }
   free(w);
   return rc;

@@ -1,0 +1,50 @@
+"""The checked build of the CUDA library (-DREGTOPK_DEBUG=1: every data-dependent index is range-checked on the
+device, a bad one is counted and skipped) run through the parity cases of every code path, in a process of its
+own so that no other test sees that library.  Parity must hold and no range check may have fired."""
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+SCRIPT = r"""
+import sys
+sys.path.insert(0, %(root)r)
+import torch
+from paper_2501_05633_b200 import binding
+binding._LIB = binding.build_checked()          # before the first load: this process uses the checked library only
+from paper_2501_05633_b200 import synth
+from tests.parity import run_parity
+from tests.test_gpu_parity import gauss_rounds
+
+WIDE, DENSE = binding.FLAG_FORCE_WIDE_LISTS, binding.FLAG_FORCE_DENSE_SELECT
+stats = []
+for (d, N, k) in [(1, 1, 1), (513, 3, 1), (4096, 8, 41), (65537, 2, 655), (200003, 2, 200003), (3001, 33, 7)]:
+    for mu in (4.0, 0.0):
+        for flags in (0, WIDE):
+            stats.append(run_parity(gauss_rounds(N, d, 3, seed=d + N), d, N, k, mu, flags=flags))
+stats.append(run_parity(gauss_rounds(3, 90_001, 4, seed=21), 90_001, 3, 900, 4.0, flags=DENSE, expect_dense=True))
+stats.append(run_parity(gauss_rounds(3, 90_001, 4, seed=21), 90_001, 3, 900, 4.0, flags=DENSE | WIDE, expect_dense=True))
+stats.append(run_parity(gauss_rounds(3, 150_000, 4, seed=8, quant=2), 150_000, 3, 1500, 4.0))
+stats.append(run_parity(gauss_rounds(2, 120_007, 4, seed=12, ld=120_008, dtype=torch.bfloat16), 120_007, 2, 1200, 4.0))
+stats.append(run_parity(gauss_rounds(3, 100_001, 4, seed=9, ld=100_004), 100_001, 3, 1000, 4.0,
+                        inplace=lambda t: t %% 2 == 1))
+for name in ("resnet18", "gpt2"):
+    w = synth.workload(name, scale_to=300_000)
+    for k in w.k_values():
+        s = synth.GradientStream(w, device="cpu", seed=17, pad_to=8)
+        stats.append(run_parity((s.next() for _ in range(6)), w.d, w.N, max(k, 1), w.mu))
+bad = [st for st in stats if st["device_error_bits"]]
+assert not bad, bad
+assert binding.library_path().endswith("libregtopk_checked.so")
+print("checked build: %%d parity runs, no range check fired" %% len(stats))
+"""
+
+
+@pytest.mark.gpu
+def test_checked_build_runs_every_path_without_a_range_fault():
+    r = subprocess.run([sys.executable, "-c", SCRIPT % {"root": ROOT}], capture_output=True, text=True, timeout=1500)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-4000:]
+    assert "no range check fired" in r.stdout
