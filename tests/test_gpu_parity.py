@@ -34,6 +34,13 @@ def test_sizes(d, N, k, mu):
     run_parity(gauss_rounds(N, d, 4, seed=d + N), d, N, k, mu)
 
 
+def test_every_tiny_size():
+    """d = 1 .. 64 with k = 1, about d/2 and d (where every entry is sent), ties included."""
+    for d in range(1, 65):
+        for k in sorted({1, max(1, d // 2), d}):
+            run_parity(gauss_rounds(2, d, 3, seed=1000 + d, quant=4 if d % 3 == 0 else 0), d, 2, k, 4.0)
+
+
 @pytest.mark.parametrize("mu", [1.0, 4.0, 10.0, 1e-30])
 def test_mu_sweep(mu):
     run_parity(gauss_rounds(4, 50_001, 5, seed=3), 50_001, 4, 500, mu)
