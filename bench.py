@@ -184,8 +184,18 @@ def cpu_baseline(w, k, seed):
     t0 = time.perf_counter()
     ora.worker_step(g1); ora.aggregate()
     el = time.perf_counter() - t0
-    return {"value": nw * w.d / el / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"one round (round 1) of {nw} of the {w.N} workers at full d={w.d}, k={k}, {el:.1f} s"}
+    out = {"value": nw * w.d / el / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": f"one round (round 1) of {nw} of the {w.N} workers at full d={w.d}, k={k}, {el:.1f} s"}
+    # second figure: the same oracle with its workers (they are independent) spread over the host's cores
+    cores = min(nw, os.cpu_count() or 1)
+    if cores > 1 and el < 60.0:
+        par = OracleRegTopK(w.d, nw, k, w.mu, threads=cores)
+        par.worker_step(g0); par.aggregate()
+        t0 = time.perf_counter()
+        par.worker_step(g1); par.aggregate()
+        el2 = time.perf_counter() - t0
+        out["workers_in_parallel"] = {"value": nw * w.d / el2 / 1e9, "unit": UNIT, "cores": cores}
+    return out
 
 
 def main():
