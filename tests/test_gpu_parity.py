@@ -208,6 +208,13 @@ def test_wide_lists_sizes(d, N, k, mu):
     run_parity(gauss_rounds(N, d, 4, seed=d + N + 1), d, N, k, mu, flags=WIDE)
 
 
+def test_wide_lists_by_size_alone():
+    """N*k large enough for the wide kernels without the flag: one worker with a long list, and a thousand
+    workers with short ones (more workers than the grid has blocks)."""
+    run_parity(gauss_rounds(1, 1_000_003, 3, seed=3, ld=1_000_008), 1_000_003, 1, 300_000, 4.0, threads=8, select_mode=1)
+    run_parity(gauss_rounds(1000, 600_000, 3, seed=0), 600_000, 1000, 300, 4.0, threads=8, select_mode=1)
+
+
 def test_wide_lists_dense_path_ties_bf16_exponent_inplace():
     run_parity(gauss_rounds(3, 90_001, 4, seed=21), 90_001, 3, 900, 4.0, flags=WIDE | binding.FLAG_FORCE_DENSE_SELECT,
                expect_dense=True)
