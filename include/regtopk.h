@@ -160,6 +160,7 @@ typedef struct {
   int64_t candidate_capacity;   /* per-worker capacity of the candidate list                              */
   int64_t device_error_bits;    /* 0, or which internal consistency check failed (1 count, 2 dense, 4 refine; 8: a
                                    range check of the checked build, -DREGTOPK_DEBUG=1) */
+  int64_t post_cluster_blocks;  /* thread blocks per worker in the selection kernel's clusters */
 } regtopk_stats;
 
 /* Synchronises the stream and fills *out (host). */

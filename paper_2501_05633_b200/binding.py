@@ -39,7 +39,8 @@ class Params(ctypes.Structure):
 class Stats(ctypes.Structure):
     _fields_ = [("rounds", ctypes.c_int64), ("kernel_launches", ctypes.c_int64),
                 ("dense_select_workers", ctypes.c_int64), ("candidates_last", ctypes.c_int64),
-                ("candidate_capacity", ctypes.c_int64), ("device_error_bits", ctypes.c_int64)]
+                ("candidate_capacity", ctypes.c_int64), ("device_error_bits", ctypes.c_int64),
+                ("post_cluster_blocks", ctypes.c_int64)]
 
 
 def library_path() -> str:

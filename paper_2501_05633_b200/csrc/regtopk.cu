@@ -1697,14 +1697,14 @@ void post_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int N, int 
   launch_config(cfg, attr, (unsigned)(N * cluster), cluster, threads, 0, s);
 }
 
-// Blocks per worker for k_post: the largest power of two up to 16 (sizes above 8 need the
+// Blocks per worker for k_post: the largest cluster size up to 16 (sizes above 8 need the
 // non-portable opt-in) for which the device keeps all N clusters resident at once; failing that,
 // the largest size it can schedule at all.
 int choose_cluster(int N) {
   cudaFuncSetAttribute(k_post, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   cudaGetLastError();
   int schedulable = 1;
-  for (int cs = kMaxCluster; cs > 1; cs >>= 1) {
+  for (int cs = kMaxCluster; cs > 1; --cs) {  // any size, not only powers of two: 10 blocks for N = 8 on a B200
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[2];
     post_config(&cfg, attr, N, cs, kBlockPost, nullptr);
@@ -2111,6 +2111,7 @@ int regtopk_get_stats(regtopk_ctx* c, regtopk_stats* out) {
     for (int n = 0; n < c->N; ++n) out->candidates_last += w[n].cand_count;
     out->candidate_capacity = c->L.capA;
     out->device_error_bits = (int64_t)h.err;
+    out->post_cluster_blocks = c->cluster;
 #if REGTOPK_DEBUG
     unsigned int faults = 0;
     if (cudaMemcpyFromSymbol(&faults, g_bounds_faults, sizeof faults) == cudaSuccess && faults)
