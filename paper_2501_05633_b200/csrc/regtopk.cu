@@ -66,6 +66,7 @@ constexpr int kBins = 4096;                // histogram bins of the select
 constexpr int kMaxCluster = 16;
 constexpr int kMaxSegments = kMaxCluster * 32;  // mask segments per row: one per warp of a k_post cluster
 constexpr u32 kFull = 0xFFFFFFFFu;
+constexpr u32 kExactRounds = 1024;  // rounds of exact cutoffs after a fallback to the dense path
 
 enum : u32 { kErrCountMismatch = 1u, kErrDenseSelect = 2u, kErrRefine = 4u, kErrBounds = 8u };
 
@@ -95,7 +96,10 @@ struct WorkerCtl {
   u32 above1;       //   exact path (written by k_wide_classify, read by k_post and k_wide_emit)
   u32 go_dense;
   u32 took_dense;   // wide mode: the dense path produced the winner list (written by k_post)
-  u32 pad[5];
+  u32 exact_rounds; // rounds for which k_sample_cutoff resolves the cutoff exactly inside its bin; set when the
+                    // selection had to fall back to the dense path, counted down by k_sample_cutoff, and kept
+                    // across rounds (nothing else resets it but regtopk_state_reset)
+  u32 pad[4];
 };
 
 struct GlobalCtl {
@@ -291,6 +295,7 @@ struct SampleArgs {
   WorkerCtl* ctl;
   u32* ghist;  // [N][4][kBins] histograms of k_post, cleared here
   u32* shist;  // [N][kSampleBins] histogram of this kernel; zero on entry (k_post clears it again)
+  u32* skeys;  // [N][kSampleMax] the sample's keys (0xFFFFFFFF in unused slots), for the exact second look
   int force_dense;
   // Clusters beyond the first N compute the regularised scores of the previous support
   // (Eq. (Delta_def), Algorithm 2 steps 8-9) while the first N sample.  On that support the
@@ -387,6 +392,9 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
     override_scores<BF16>(p, (int64_t)blockIdx.x * blockDim.x + tid, (int64_t)gridDim.x * blockDim.x);
   WorkerCtl* ctl = p.ctl + n;
   u32* shist = p.shist + (size_t)n * kSampleBins;
+  // exact cutoff wanted this round (see below)?  Read by every thread of the cluster here, long before the
+  // leader's thread 0 counts it down behind the cluster barrier.
+  const bool want_exact = ctl->exact_rounds != 0u;
 
   for (int i = rk * blockDim.x + tid; i < 4 * kBins; i += kSampleCluster * blockDim.x)
     p.ghist[(size_t)n * 4 * kBins + i] = 0;
@@ -428,8 +436,11 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
     for (int i = tid; i < kSamplePadded; i += blockDim.x) s_hist[i] = 0;  // while the loads are in flight
     __syncthreads();
 #pragma unroll
-    for (int u = 0; u < 8; ++u)
-      if (ok[u]) atomicAdd(&s_hist[sample_slot((__float_as_uint(p.inplace ? e[u] : __fadd_rn(e[u], g[u])) & 0x7FFFFFFFu) >> kSampleShift)], 1u);
+    for (int u = 0; u < 8; ++u) {
+      const u32 key = __float_as_uint(p.inplace ? e[u] : __fadd_rn(e[u], g[u])) & 0x7FFFFFFFu;
+      if (want_exact) p.skeys[(size_t)n * kSampleMax + (int)rk * kSamplePerBlock + u * kBlockSel + tid] = ok[u] ? key : kFull;
+      if (ok[u]) atomicAdd(&s_hist[sample_slot(key >> kSampleShift)], 1u);
+    }
   }
   __syncthreads();
   for (int i = tid; i < kSampleBins; i += blockDim.x) {
@@ -487,16 +498,47 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
   // the cutoff: inside the bin that holds the r_lo-th largest sample, placed as if the bin's sample
   // points were spread evenly over it (0: keep everything).  Error feedback piles entries up just
   // below the selection threshold, so a cutoff a whole bin too low would gather far too many.
+  // Error feedback can pack a large part of a row into a band much narrower than a bin, right under the
+  // selection threshold; that guess can then land above the whole band and leave fewer than k entries
+  // above the cutoff (or below it and gather far too many).  The selection notices (it falls back to its dense
+  // path, which is exact but slow) and asks for the next rounds' cutoffs to be resolved exactly: the sample's keys
+  // are then read once more and the position inside the bin is found down to 32 key units (about 5 us more).
   u32 cutoff = 0u;
   if (r_lo <= (u32)M && s_res[1] != kFull) {
     const u32 width = 1u << kSampleShift;
-    const u32 below = (u32)(((u64)(s_frac[0] - s_frac[1]) * width) / (s_frac[0] + 1u));  // offset from the bin's lower edge
-    cutoff = (s_res[1] << kSampleShift) + below;
+    const u32 bin = s_res[1], in_bin = s_frac[0], need = s_frac[1];  // the same in every thread
+    if (want_exact) {
+      __syncthreads();  // every thread has read s_res / s_frac and its bins of s_hist
+      for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
+      __syncthreads();
+      const u32* keys = p.skeys + (size_t)n * kSampleMax;
+      const uint4* keys4 = reinterpret_cast<const uint4*>(keys);
+      for (int i0 = 0; i0 < kSampleMax / 4; i0 += 8 * kBlockSel) {  // two rounds of eight 16-byte loads per thread
+        uint4 kk[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) kk[q] = __ldcg(&keys4[i0 + q * kBlockSel + tid]);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const u32 v[4] = {kk[q].x, kk[q].y, kk[q].z, kk[q].w};
+#pragma unroll
+          for (int z = 0; z < 4; ++z)
+            if ((v[z] >> kSampleShift) == bin) atomicAdd(&s_hist[(v[z] >> (kSampleShift - 12)) & (u32)(kBins - 1)], 1u);
+        }
+      }
+      __syncthreads();
+      block_find_from_top(s_hist, kBins, need, s_scan, s_res);  // the sub-bin of the need-th largest key of the bin
+      const u32 sub = s_res[0] == kFull ? 0u : s_res[0];
+      cutoff = (bin << kSampleShift) + (sub << (kSampleShift - 12));
+    } else {
+      const u32 below = (u32)(((u64)(in_bin - need) * width) / (in_bin + 1u));  // offset from the bin's lower edge
+      cutoff = (bin << kSampleShift) + below;
+    }
   }
   if (tid == 0) {
     const u32 range = hi_key > cutoff ? hi_key - cutoff : 0u;
     u32 shift = 0;
     while ((range >> shift) > (u32)(kBins - 2)) ++shift;
+    if (want_exact) ctl->exact_rounds -= 1u;
     ctl->cutoff = cutoff;
     ctl->bin_shift = shift;
     ctl->cand_count = 0;
@@ -1130,7 +1172,10 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
     if (!dense) {
       load_and_find(sh, ghist, k, &b1, &above1, &nvalid);
       if (b1 == kFull || overflow) dense = true;  // cutoff guessed too high, or the list overflowed
-      if (rk == 0 && tid == 0) ctl->n_valid = nvalid;
+      if (rk == 0 && tid == 0) {
+        ctl->n_valid = nvalid;
+        if (dense) ctl->exact_rounds = kExactRounds;
+      }
     }
     if (!dense) {
       post_classify(p, n, first_t, stride_t, ncand, novr, cutoff, bshift, b1);
@@ -1296,6 +1341,7 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_wide_classify
     ctl->above1 = above1;
     ctl->go_dense = dense ? 1u : 0u;
     ctl->n_valid = nvalid;
+    if (dense && ctl->force_dense == 0) ctl->exact_rounds = kExactRounds;
   }
   if (!dense) post_classify(p, n, first_t, stride_t, ncand, p.use_marks ? (u32)p.k : 0u, cutoff, bshift, b1);
 }
@@ -1538,7 +1584,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   int64_t ld, W, capA, stride;
-  size_t off_eps, off_g, off_mask[2], off_ctl, off_gctl, off_shist, zero_end, off_qprefix, off_segtot, off_segbase, off_ghist, off_btot, off_idx[2], off_val[2],
+  size_t off_eps, off_g, off_mask[2], off_ctl, off_gctl, off_shist, zero_end, off_skeys, off_qprefix, off_segtot, off_segbase, off_ghist, off_btot, off_idx[2], off_val[2],
       off_ovr_key, off_ovr_comp, off_candA, off_candB, off_omega, off_stage_g, off_stage_idx,
       off_stage_val, total;
 };
@@ -1577,6 +1623,7 @@ Layout make_layout(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
   L.off_gctl = take(sizeof(GlobalCtl));
   L.off_shist = take((size_t)N * kSampleBins * 4);
   L.zero_end = o;
+  L.off_skeys = take((size_t)N * kSampleMax * 4);
   L.off_qprefix = take((size_t)N * (L.W / 4) * 4);
   L.off_segtot = take((size_t)N * kMaxSegments * 4);
   L.off_segbase = take((size_t)N * kMaxSegments * 4);
@@ -1827,6 +1874,7 @@ int step_impl(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_i
   sa.k_target = use_marks ? (2 * c->k < c->d ? 2 * c->k : c->d) : c->k;
   sa.ctl = at<WorkerCtl>(c, L.off_ctl);
   sa.shist = at<u32>(c, L.off_shist);
+  sa.skeys = at<u32>(c, L.off_skeys);
   sa.ghist = at<u32>(c, L.off_ghist);
   sa.N = c->N; sa.use_marks = use_marks; sa.g_prev = at<float>(c, L.off_g);
   sa.prev_idx = at<int32_t>(c, L.off_idx[prev]); sa.prev_val = at<float>(c, L.off_val[prev]);

@@ -281,6 +281,25 @@ def test_long_run_stays_exact_and_on_the_fast_path():
     assert st["dense_select_workers"] == 0, st
 
 
+def test_pile_up_under_the_threshold_does_not_keep_the_dense_path():
+    """Thousands of rounds on a short cycle of batches: error feedback packs the unsent entries into a band right
+    under the selection threshold that is far narrower than a bin of the cutoff sample.  A cutoff placed by
+    interpolation then misses; after the first fallback the library resolves its cutoffs exactly, so the dense
+    path stays the exception (once per worker and 1024 rounds at most)."""
+    w = synth.workload("gpt2", scale_to=2_000_000)
+    k = w.k_values()[0]
+    s = synth.GradientStream(w, device="cuda", seed=8, pad_to=32)
+    ring = [s.next() for _ in range(8)]
+    lib = RegTopK(w.d, w.N, k, mu=w.mu, grad_dtype=torch.bfloat16)
+    rounds = 6000
+    for t in range(rounds):
+        lib.worker_step(ring[t % 8])
+        lib.aggregate()
+    lib.status()
+    st = lib.stats()
+    assert st["dense_select_workers"] <= w.N * (rounds // 1024 + 2), st
+
+
 def test_least_squares_trajectory():
     """N=8, 512x4096 least squares, k=41, 100 rounds with step 0.1: identical masks, residuals and
     aggregates every round, hence the identical loss curve, which must fall."""
