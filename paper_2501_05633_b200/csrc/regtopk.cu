@@ -66,7 +66,16 @@ constexpr int kBins = 4096;                // histogram bins of the select
 constexpr int kMaxCluster = 16;
 constexpr int kMaxSegments = kMaxCluster * 32;  // mask segments per row: one per warp of a k_post cluster
 constexpr u32 kFull = 0xFFFFFFFFu;
-constexpr u32 kExactRounds = 1024;  // rounds of exact cutoffs after a fallback to the dense path
+constexpr u32 kExactRounds = 1024;     // rounds of exact cutoffs after a first fallback to the dense path;
+constexpr u32 kExactRoundsMax = 1u << 20;  // doubled after every further one, up to this
+
+// One thread, after its worker fell back to the dense path because the cutoff was off.
+__device__ __forceinline__ void ask_for_exact_cutoffs(volatile u32* exact_rounds, volatile u32* exact_window) {
+  const u32 w = *exact_window;
+  const u32 next = w == 0u ? kExactRounds : (w >= kExactRoundsMax / 2u ? kExactRoundsMax : 2u * w);
+  *exact_window = next;
+  *exact_rounds = next;
+}
 
 enum : u32 { kErrCountMismatch = 1u, kErrDenseSelect = 2u, kErrRefine = 4u, kErrBounds = 8u };
 
@@ -99,7 +108,8 @@ struct WorkerCtl {
   u32 exact_rounds; // rounds for which k_sample_cutoff resolves the cutoff exactly inside its bin; set when the
                     // selection had to fall back to the dense path, counted down by k_sample_cutoff, and kept
                     // across rounds (nothing else resets it but regtopk_state_reset)
-  u32 pad[4];
+  u32 exact_window; // length of the last such stretch: it doubles with every further fallback
+  u32 pad[3];
 };
 
 struct GlobalCtl {
@@ -125,6 +135,22 @@ __device__ __forceinline__ u32 composite_idx(u64 c) { return kFull - static_cast
 // ---------------------------------------------------------------------------------------------
 // block-wide helpers (blockDim.x a multiple of 32, at most 1024)
 // ---------------------------------------------------------------------------------------------
+
+// Histogram increment for data that may pile up in one bin (error feedback packs the entries under the
+// selection threshold into a narrow band): when all lanes of a warp that have an item hit the same bin, one of
+// them adds the count; otherwise every lane adds its own.  Every lane of the warp must call it (pred: this
+// lane has an item).
+__device__ __forceinline__ void hist_add_aggregated(u32* hist, bool pred, u32 bin) {
+  const u32 act = __ballot_sync(kFull, pred);
+  if (act == 0u) return;
+  const int first = __ffs(act) - 1;
+  const u32 bin0 = __shfl_sync(kFull, bin, first);
+  if (__all_sync(kFull, !pred || bin == bin0)) {
+    if ((int)(threadIdx.x & 31) == first) atomicAdd(&hist[bin0], (u32)__popc(act));
+  } else if (pred) {
+    atomicAdd(&hist[bin], 1u);
+  }
+}
 
 // Exclusive prefix sum of v over the block in thread order; *total receives the block sum.
 // s_scan: 33 words of shared memory.  Every thread of the block must call it.
@@ -1174,7 +1200,7 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
       if (b1 == kFull || overflow) dense = true;  // cutoff guessed too high, or the list overflowed
       if (rk == 0 && tid == 0) {
         ctl->n_valid = nvalid;
-        if (dense) ctl->exact_rounds = kExactRounds;
+        if (dense) ask_for_exact_cutoffs(&ctl->exact_rounds, &ctl->exact_window);
       }
     }
     if (!dense) {
@@ -1189,6 +1215,49 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
     if (nB <= blockDim.x) {
       // every block ranks the short list itself and sets the winners of its own share of the mask
       refine_small(sh, mask, p.d, B, nB, need, su0 * 8, su1 * 8);
+    } else if (nB <= k) {
+      // A crowded threshold bin (error feedback packs the entries under the threshold into a band that a few
+      // bins cover): a second histogram over that bin's own key range, 4096 sub-bins, by the whole cluster;
+      // what is left in the sub-bin of the threshold (keys equal or nearly so) goes to the list refinement.
+      // The second list lives behind the candidates in A (k entries are free there).
+      const u32 lo2 = cutoff + (b1 << bshift);  // lower edge of the threshold bin; every listed key is at or above it
+      u32 shift2 = bshift > 12u ? bshift - 12u : 0u;
+      if (b1 == (u32)(kBins - 1)) {  // the clamped top bin reaches up to the largest key
+        shift2 = 0;
+        while (((0x7FFFFFFFu - lo2) >> shift2) > (u32)(kBins - 2)) ++shift2;
+      }
+      u64* B2 = A + p.capA;
+      __syncthreads();
+      for (int i = tid; i < kBins; i += blockDim.x) sh.hist[i] = 0;
+      __syncthreads();
+      for (u32 i = first_t; i < nB; i += stride_t)
+        atomicAdd(&sh.hist[select_bin((u32)(__ldcg(B + i) >> 32), lo2, shift2)], 1u);
+      __syncthreads();
+      flush_hist(sh.hist, ghist + kBins, kBins);  // the second of the four histograms: unused on this path so far
+      cl.sync();  // (2c) histogram of the threshold bin complete
+      u32 b2, above2, total2;
+      load_and_find(sh, ghist + kBins, need, &b2, &above2, &total2);  // need <= nB: always found
+      const u32 iters2 = (nB + stride_t - 1) / stride_t;
+      for (u32 it = 0; it < iters2; ++it) {
+        const u32 i = it * stride_t + first_t;
+        const u64 c = i < nB ? __ldcg(B + i) : 0ull;
+        const u32 sub = c ? select_bin((u32)(c >> 32), lo2, shift2) : 0u;
+        if (c && b2 != kFull && sub > b2) set_winner(mask, composite_idx(c), p.d);
+        const bool inb = c && sub == b2;
+        const u32 pos = warp_reserve_global(inb, &ctl->acount);  // acount: otherwise the dense path's counter
+        if (inb && RT_INB(pos < k)) B2[pos] = c;
+      }
+      cl.sync();  // (2d) second list complete
+      const u32 nB2 = __ldcg(&ctl->acount);
+      const u32 need2 = need - above2;
+      if (b2 == kFull) {
+        if (rk == 0 && tid == 0) atomicOr(&p.gctl->err, kErrRefine);  // cannot happen while need <= nB
+      } else if (nB2 <= blockDim.x) {
+        refine_small(sh, mask, p.d, B2, nB2, need2, su0 * 8, su1 * 8);
+      } else {
+        if (rk == 0) refine_large(sh, mask, p.d, p.gctl, B2, nB2, need2);
+        cl.sync();  // (2e) the leader's winners are set
+      }
     } else {
       if (rk == 0) refine_large(sh, mask, p.d, p.gctl, B, nB, need);
       cl.sync();  // (2b) the leader's winners are set
@@ -1209,9 +1278,11 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
       __syncthreads();
       for (int i = tid; i < kBins; i += blockDim.x) sh.hist[i] = 0;
       __syncthreads();
-      for (int64_t j = c0 + tid; j < c1; j += blockDim.x) {
-        const u32 key = dense_key(p, n, j);
-        if (lv == 0 || (key >> (shf + widths[lv])) == prefix) atomicAdd(&sh.hist[(key >> shf) & nbm], 1u);
+      for (int64_t base = c0; base < c1; base += blockDim.x) {  // whole warps iterate: the increments are aggregated
+        const int64_t j = base + tid;
+        const u32 key = j < c1 ? dense_key(p, n, j) : 0u;
+        const bool in = j < c1 && (lv == 0 || (key >> (shf + widths[lv])) == prefix);
+        hist_add_aggregated(sh.hist, in, (key >> shf) & nbm);  // rows that end up here are full of equal digits
       }
       __syncthreads();
       flush_hist(sh.hist, ghist + (1 + lv) * kBins, kBins);
@@ -1341,7 +1412,7 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_wide_classify
     ctl->above1 = above1;
     ctl->go_dense = dense ? 1u : 0u;
     ctl->n_valid = nvalid;
-    if (dense && ctl->force_dense == 0) ctl->exact_rounds = kExactRounds;
+    if (dense && ctl->force_dense == 0) ask_for_exact_cutoffs(&ctl->exact_rounds, &ctl->exact_window);
   }
   if (!dense) post_classify(p, n, first_t, stride_t, ncand, p.use_marks ? (u32)p.k : 0u, cutoff, bshift, b1);
 }
