@@ -909,6 +909,22 @@ __device__ __forceinline__ u32 dense_key(const PostArgs& p, int n, int64_t j) {
   return __float_as_uint(p.eps[(size_t)n * p.ld + j]) & 0x7FFFFFFFu;
 }
 
+// The same for the four entries j4 .. j4 + 3 (j4 a multiple of 4; rows are 16-byte aligned and padded): one
+// 16-byte load of the residuals and one mask word; only entries on the previous support, which are few, take the
+// search.  Keys of entries at or beyond `end` are 0 and not to be used.
+__device__ __forceinline__ void dense_keys4(const PostArgs& p, int n, int64_t j4, int64_t end, u32 (&key)[4]) {
+  key[0] = key[1] = key[2] = key[3] = 0u;
+  if (j4 >= end) return;
+  const float4 e = *reinterpret_cast<const float4*>(p.eps + (size_t)n * p.ld + j4);
+  const u32 w = p.use_marks ? (p.mask_old[(size_t)n * p.W + (j4 >> 5)] >> (j4 & 31)) & 15u : 0u;
+  const float v[4] = {e.x, e.y, e.z, e.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    if (j4 + q >= end) break;
+    key[q] = ((w >> q) & 1u) ? dense_key(p, n, j4 + q) : (__float_as_uint(v[q]) & 0x7FFFFFFFu);
+  }
+}
+
 // One block: among list[0..count) (count <= blockDim.x, unique composites) set the `need` largest as
 // winners, but only those whose mask word lies in [w0, w1) (the caller's share of the mask).
 __device__ void refine_small(PostShared& sh, u32* mask, int64_t d, const u64* list, u32 count, u32 need,
@@ -1266,8 +1282,9 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
     // ---- exact selection over the whole row: three radix digits of the 31-bit key ----
     took_dense = true;
     if (rk == 0 && tid == 0) atomicAdd(&p.gctl->dense_workers, 1ull);
-    const int64_t c0 = (int64_t)(((u64)rk * (u64)p.d) / CS);
-    const int64_t c1 = (int64_t)(((u64)(rk + 1) * (u64)p.d) / CS);
+    // this block's part of the row; the cuts are multiples of four so that every thread reads whole quads
+    const int64_t c0 = (int64_t)(((u64)rk * (u64)p.d) / CS) & ~(int64_t)3;
+    const int64_t c1 = rk + 1 == CS ? p.d : (int64_t)(((u64)(rk + 1) * (u64)p.d) / CS) & ~(int64_t)3;
     u32 need = k, prefix = 0;
     bool bad = false;
     const int shifts[3] = {19, 7, 0};
@@ -1278,11 +1295,15 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
       __syncthreads();
       for (int i = tid; i < kBins; i += blockDim.x) sh.hist[i] = 0;
       __syncthreads();
-      for (int64_t base = c0; base < c1; base += blockDim.x) {  // whole warps iterate: the increments are aggregated
-        const int64_t j = base + tid;
-        const u32 key = j < c1 ? dense_key(p, n, j) : 0u;
-        const bool in = j < c1 && (lv == 0 || (key >> (shf + widths[lv])) == prefix);
-        hist_add_aggregated(sh.hist, in, (key >> shf) & nbm);  // rows that end up here are full of equal digits
+      for (int64_t base = c0; base < c1; base += 4 * (int64_t)blockDim.x) {  // whole warps iterate: the increments are aggregated
+        const int64_t j4 = base + 4 * tid;
+        u32 key[4];
+        dense_keys4(p, n, j4, c1, key);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const bool in = j4 + q < c1 && (lv == 0 || (key[q] >> (shf + widths[lv])) == prefix);
+          hist_add_aggregated(sh.hist, in, (key[q] >> shf) & nbm);  // rows that end up here are full of equal digits
+        }
       }
       __syncthreads();
       flush_hist(sh.hist, ghist + (1 + lv) * kBins, kBins);
@@ -1297,17 +1318,17 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
     const u32 n_gt = k - need;     // entries strictly above it; `need` ties are to be taken
     // entries above T in any order, and this block's count of ties
     u32 my_ties = 0;
-    for (int64_t base = c0; base < c1; base += blockDim.x) {
-      const int64_t j = base + tid;
-      u32 key = 0;
-      bool gt = false;
-      if (j < c1) {
-        key = dense_key(p, n, j);
-        gt = key > T;
-        my_ties += key == T ? 1u : 0u;
+    for (int64_t base = c0; base < c1; base += 4 * (int64_t)blockDim.x) {
+      const int64_t j4 = base + 4 * tid;
+      u32 key[4];
+      dense_keys4(p, n, j4, c1, key);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const bool gt = j4 + q < c1 && key[q] > T;
+        my_ties += (j4 + q < c1 && key[q] == T) ? 1u : 0u;
+        const u32 pos = warp_reserve_global(gt, &ctl->acount);
+        if (gt && pos < n_gt) A[pos] = make_composite(key[q], (u32)(j4 + q));
       }
-      const u32 pos = warp_reserve_global(gt, &ctl->acount);
-      if (gt && pos < n_gt) A[pos] = make_composite(key, (u32)j);
     }
     u32 block_ties;
     block_excl_scan(my_ties, sh.scan, &block_ties);
@@ -1321,12 +1342,22 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
     }
     if (all_ties < need) bad = true;
     // ties in index order: the first `need` of them
-    for (int64_t base = c0; base < c1 && taken < need; base += blockDim.x) {
-      const int64_t j = base + tid;
-      const bool tie = j < c1 && dense_key(p, n, j) == T;
+    for (int64_t base = c0; base < c1 && taken < need; base += 4 * (int64_t)blockDim.x) {
+      const int64_t j4 = base + 4 * tid;  // threads hold consecutive quads: thread order is index order
+      u32 key[4];
+      dense_keys4(p, n, j4, c1, key);
+      u32 mine = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) mine += (j4 + q < c1 && key[q] == T) ? 1u : 0u;
       u32 total;
-      const u32 rank = taken + block_excl_scan(tie ? 1u : 0u, sh.scan, &total);
-      if (tie && rank < need && RT_INB(n_gt + rank < k)) A[n_gt + rank] = make_composite(T, (u32)j);
+      u32 rank = taken + block_excl_scan(mine, sh.scan, &total);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (j4 + q < c1 && key[q] == T) {
+          if (rank < need && RT_INB(n_gt + rank < k)) A[n_gt + rank] = make_composite(T, (u32)(j4 + q));
+          ++rank;
+        }
+      }
       taken += total;
     }
     cl.sync();  // winner list complete
