@@ -46,6 +46,9 @@ def _bind(path):
     L.regtopk_oracle_worker_step.restype = ctypes.c_int
     L.regtopk_oracle_worker_step.argtypes = [_c_i64, _c_i64, _vp, ctypes.c_int, _vp, _c_i64, _vp,
                                              _vp, _vp, _c_f32, _c_f32, _c_f32, _vp, _vp, ctypes.c_int]
+    L.regtopk_oracle_worker_step_layered.restype = ctypes.c_int
+    L.regtopk_oracle_worker_step_layered.argtypes = [_c_i64, _c_i64, _vp, _vp, _vp, ctypes.c_int, _vp, _c_i64, _vp,
+                                                     _vp, _vp, _c_f32, _c_f32, _c_f32, _vp, _vp]
     L.regtopk_oracle_aggregate.restype = None
     L.regtopk_oracle_aggregate.argtypes = [_c_i64, _c_i32, _c_i64, _vp, _vp, _vp, _vp]
     L.regtopk_oracle_model_update.restype = None
@@ -127,6 +130,24 @@ class OracleAPI:
             raise ValueError("oracle rejected the arguments (need 1 <= k <= d < 2^31, 0 < y <= 1)")
         return out_idx, out_val
 
+    def worker_step_layered(self, grad, eps, seg_end, seg_k, prev_idx, prev_val, g_prev, mu, omega_n, y=1.0):
+        """One worker, one round, with one Top-k per layer: layer l is [seg_end[l-1], seg_end[l]) and keeps seg_k[l]
+        entries.  eps is updated in place.  Returns (idx, val) with sum(seg_k) pairs in ascending index order."""
+        grad, code = _grad_view(grad)
+        d = grad.shape[0]
+        assert eps.dtype == np.float32 and eps.flags.c_contiguous and eps.shape == (d,)
+        se = np.ascontiguousarray(seg_end, dtype=np.int64)
+        sk = np.ascontiguousarray(seg_k, dtype=np.int64)
+        K = int(sk.sum())
+        out_idx = np.empty(K, np.int32)
+        out_val = np.empty(K, np.float32)
+        n_prev, pi, pv, gp = _prev_views(prev_idx, prev_val, g_prev)
+        rc = self.L.regtopk_oracle_worker_step_layered(d, se.shape[0], _p(se), _p(sk), _p(grad), code, _p(eps), n_prev,
+                                                       _p(pi), _p(pv), _p(gp), mu, omega_n, y, _p(out_idx), _p(out_val))
+        if rc != 0:
+            raise ValueError("oracle rejected the layer table (ascending ends, last == d, 1 <= k_l <= layer size)")
+        return out_idx, out_val
+
     def aggregate(self, d, omega, idx, val):
         idx = np.ascontiguousarray(idx, dtype=np.int32)
         val = np.ascontiguousarray(val, dtype=np.float32)
@@ -176,9 +197,14 @@ class OracleRegTopK:
     independent workers over host threads; each worker's computation is unchanged.
     """
 
-    def __init__(self, d, N, k, mu, omega=None, select_mode=0, threads=1, api=None, y=1.0):
+    def __init__(self, d, N, k, mu, omega=None, select_mode=0, threads=1, api=None, y=1.0, layers=None):
+        """layers: None, or (seg_end, seg_k) for one Top-k per layer; k is then ignored and becomes sum(seg_k)."""
         self.api = api or default()
         self.y = float(y)
+        self.layers = None
+        if layers is not None:
+            self.layers = (np.asarray(layers[0], np.int64).copy(), np.asarray(layers[1], np.int64).copy())
+            k = int(self.layers[1].sum())
         self.d, self.N, self.k, self.mu = int(d), int(N), int(k), float(mu)
         self.omega = (np.full(N, np.float32(1.0) / np.float32(N), np.float32) if omega is None
                       else np.asarray(omega, np.float32).copy())
@@ -198,6 +224,9 @@ class OracleRegTopK:
     def _one(self, n, grads):
         pi = None if self.prev_idx is None else self.prev_idx[n]
         pv = None if self.prev_val is None else self.prev_val[n]
+        if self.layers is not None:
+            return self.api.worker_step_layered(grads[n], self.eps[n], self.layers[0], self.layers[1], pi, pv,
+                                                self.g_prev, self.mu, float(self.omega[n]), self.y)
         return self.api.worker_step(grads[n], self.eps[n], self.k, pi, pv, self.g_prev, self.mu,
                            float(self.omega[n]), self.select_mode, self.y)
 

@@ -16,6 +16,8 @@
 //   residual          eps' = a - ghat                               Algorithm 1 step 7, Algorithm 2 step 12
 //   server            g = sum_n w_n * ghat_n                        Section 2.2 (aggregation equation)
 //   model update      theta' = theta - eta * g                      Section 1 (after Eq. (1))
+//   layer-wise masks  Top_{k_l} applied to each layer's slice of the score vector (the layer-wise
+//                     sparsification the paper's "Further Related Work" points to); everything else as above
 //
 // Readings taken where the paper is silent (each listed in the design notes):
 //   * ties in the magnitude sort: the lower index wins;
@@ -27,6 +29,8 @@
 //   * every operation is an individually rounded IEEE binary32 operation in the written order
 //     (compile with -ffp-contract=off; never -ffast-math).
 //
+//   * layer-wise selection: the model vector is cut into contiguous layers, layer l keeps its k_l best entries
+//     by the same ranking, and the pairs of all layers are emitted together in ascending index order;
 // Pins (tests/test_oracle_*.py): brute force over all subsets on tiny inputs; k = d pass-through;
 // round 0 / mu = 0 / mu -> 0 against an independent Top-k with error feedback; the error-feedback
 // identity; the toy logistic example (Delta = -1 exactly); the printed iteration-1 column of the
@@ -235,6 +239,49 @@ int regtopk_oracle_worker_step(int64_t d, int64_t k, const void* grad, int grad_
     out_idx[i] = j;
     out_val[i] = a[j];  // the raw accumulator, not the score
     eps[j] = 0.0f;      // a - a
+  }
+  return 0;
+}
+
+// Layer-wise form of the same round: the d coordinates are cut into n_seg contiguous layers, layer l being
+// [seg_end[l-1], seg_end[l]) (seg_end ascending, seg_end[n_seg-1] == d), and the mask is the union over the layers
+// of Top_{seg_k[l]} of the score restricted to that layer (1 <= seg_k[l] <= the layer's size).  Accumulator, posterior
+// distortion, regulariser, sent values and residual are those of regtopk_oracle_worker_step; only the selector
+// changes.  out_idx/out_val receive sum_l seg_k[l] pairs in ascending index order.  Selection by a full sort of
+// each layer's records.  Returns 0, or -1 on invalid sizes.
+int regtopk_oracle_worker_step_layered(int64_t d, int64_t n_seg, const int64_t* seg_end, const int64_t* seg_k,
+                                       const void* grad, int grad_dtype, float* eps, int64_t n_prev,
+                                       const int32_t* prev_idx, const float* prev_val, const float* g_prev,
+                                       float mu, float omega_n, float y, int32_t* out_idx, float* out_val) {
+  if (d < 1 || d > INT32_MAX || n_seg < 1 || !(y > 0.0f && y <= 1.0f)) return -1;
+  int64_t begin = 0;
+  for (int64_t l = 0; l < n_seg; ++l) {
+    if (seg_end[l] <= begin || seg_k[l] < 1 || seg_k[l] > seg_end[l] - begin) return -1;
+    begin = seg_end[l];
+  }
+  if (begin != d) return -1;
+  std::vector<float> a(d), score(d);
+  regtopk_oracle_scores(d, grad, grad_dtype, eps, n_prev, prev_idx, prev_val, g_prev, mu, omega_n, y,
+                        a.data(), score.data());
+  for (int64_t j = 0; j < d; ++j) eps[j] = a[j];  // (a minus 0 wherever no layer sends the entry)
+  int64_t out = 0;
+  begin = 0;
+  for (int64_t l = 0; l < n_seg; ++l) {
+    const int64_t end = seg_end[l], kl = seg_k[l];
+    std::vector<Scored> rec;
+    for (int64_t j = begin; j < end; ++j) rec.push_back(Scored{score[j], static_cast<int32_t>(j)});
+    std::sort(rec.begin(), rec.end(), ranks_before);
+    std::vector<int32_t> chosen(kl);
+    for (int64_t i = 0; i < kl; ++i) chosen[i] = rec[i].idx;
+    std::sort(chosen.begin(), chosen.end());
+    for (int64_t i = 0; i < kl; ++i) {
+      int32_t j = chosen[i];
+      out_idx[out] = j;      // layers are index ranges in ascending order, so the whole output ascends
+      out_val[out] = a[j];   // the raw accumulator, not the score
+      eps[j] = 0.0f;         // a - a
+      ++out;
+    }
+    begin = end;
   }
   return 0;
 }

@@ -393,7 +393,103 @@ def pin_mask_certificate(api):
     assert api.mask_certificate(s, wrong) != k
 
 
-ALL_PINS = [pin_tanh, pin_bruteforce_selector, pin_dense_passthrough, pin_reduces_to_topk,
+def _random_layers(rng, d, max_layers):
+    n_seg = int(rng.integers(1, min(max_layers, d) + 1))
+    cuts = np.sort(rng.choice(np.arange(1, d), size=n_seg - 1, replace=False)) if n_seg > 1 else np.array([], np.int64)
+    seg_end = np.concatenate([cuts, [d]]).astype(np.int64)
+    sizes = np.diff(np.concatenate([[0], seg_end]))
+    seg_k = np.array([int(rng.integers(1, sz + 1)) for sz in sizes], np.int64)
+    return seg_end, seg_k
+
+
+def pin_layered_bruteforce(api):
+    """One Top-k per layer, by enumeration: in every layer the chosen set is the best k_l-subset of that layer's
+    indices (descending score tuple, then ascending index tuple); all layers' pairs come out in ascending index
+    order with the raw accumulator as value; the residual is cleared exactly there."""
+    rng = np.random.default_rng(17)
+    for trial in range(60):
+        d = int(rng.integers(2, 10))
+        g = rng.choice(np.array([0.0, 0.0, 0.5, -0.5, 1.0, -1.0, 2.0, 3.5, -3.5], np.float32), size=d).astype(np.float32)
+        eps0 = rng.choice(np.array([0.0, 0.0, 0.25, -1.0], np.float32), size=d).astype(np.float32)
+        if trial % 2 == 1:
+            kp = int(rng.integers(1, d + 1))
+            pidx = np.sort(rng.choice(d, size=kp, replace=False)).astype(np.int32)
+            pval = rng.choice(np.array([0.5, -1.0, 2.0, 4.0], np.float32), size=kp).astype(np.float32)
+            gprev = rng.choice(np.array([0.0, 0.5, -1.0, 2.0], np.float32), size=d).astype(np.float32)
+            eps0[pidx] = 0.0
+        else:
+            pidx = pval = gprev = None
+        seg_end, seg_k = _random_layers(rng, d, 4)
+        a, s = api.scores(g, eps0, pidx, pval, gprev, 2.0, 0.5)
+        eps = eps0.copy()
+        idx, val = api.worker_step_layered(g, eps, seg_end, seg_k, pidx, pval, gprev, 2.0, 0.5)
+        want = []
+        begin = 0
+        for end, kl in zip(seg_end, seg_k):
+            best = None
+            for sub in itertools.combinations(range(begin, int(end)), int(kl)):
+                key = (tuple(sorted((-float(s[j]) for j in sub))), sub)
+                if best is None or key < best:
+                    best = key
+            want += list(best[1])
+            begin = int(end)
+        assert [int(i) for i in idx] == want, (d, seg_end, seg_k, s, idx, want)
+        assert np.array_equal(val, a[idx])
+        expect_eps = a.copy()
+        expect_eps[idx] = 0.0
+        assert np.array_equal(eps.view(np.uint32), expect_eps.view(np.uint32))
+
+
+def pin_layered_special_cases(api):
+    """(i) One layer covering everything is the global selector.  (ii) k_l equal to the layer's size sends the whole
+    layer.  (iii) A layer's mask depends only on that layer's scores: it equals Algorithm 1 (independent numpy
+    Top-k) applied to the layer's slice alone, in round 0, for several rounds of error feedback with mu = 0."""
+    rng = np.random.default_rng(23)
+    d, N = 300, 2
+    rounds = [np.round(rng.standard_normal((N, d)) * 8).astype(np.float32) / 8 for _ in range(5)]  # ties included
+    # (i)
+    G = OracleRegTopK(d, N, 37, 4.0, api=api)
+    L1 = OracleRegTopK(d, N, 0, 4.0, api=api, layers=([d], [37]))
+    for g in rounds:
+        ig, vg = G.worker_step(g)
+        il, vl = L1.worker_step(g)
+        assert np.array_equal(ig, il) and np.array_equal(vg, vl) and np.array_equal(G.eps, L1.eps)
+        assert np.array_equal(G.aggregate(), L1.aggregate())
+    # (ii) and (iii)
+    seg_end = np.array([40, 41, 170, 300], np.int64)
+    seg_k = np.array([40, 1, 13, 7], np.int64)
+    omega = np.full(N, 0.5, np.float32)
+    refs = []
+    begin = 0
+    for end, kl in zip(seg_end, seg_k):
+        refs.append(topk_error_feedback_numpy([g[:, begin:end] for g in rounds], int(kl), omega))
+        begin = int(end)
+    O = OracleRegTopK(d, N, 0, 0.0, omega=omega, api=api, layers=(seg_end, seg_k))
+    for t, g in enumerate(rounds):
+        idx, val = O.worker_step(g)
+        agg = O.aggregate()
+        assert np.array_equal(idx[:, :40], np.tile(np.arange(40, dtype=np.int32), (N, 1)))  # (ii)
+        begin, col = 0, 0
+        for l, (end, kl) in enumerate(zip(seg_end, seg_k)):
+            ri, rv, reps, ragg = refs[l][t]
+            assert np.array_equal(idx[:, col:col + kl] - begin, ri), (t, l)
+            assert np.array_equal(val[:, col:col + kl], rv)
+            assert np.array_equal(O.eps[:, begin:end], reps)
+            assert np.array_equal(agg[begin:end], ragg)
+            begin, col = int(end), col + int(kl)
+
+
+def pin_layered_rejects_bad_tables(api):
+    g = np.ones(10, np.float32)
+    for seg_end, seg_k in (([5, 9], [1, 1]), ([5, 5, 10], [1, 1, 1]), ([4, 10], [5, 1]), ([4, 10], [0, 1]), ([10, 4], [1, 1])):
+        try:
+            api.worker_step_layered(g, np.zeros(10, np.float32), seg_end, seg_k, None, None, None, 4.0, 0.5)
+        except ValueError:
+            continue
+        raise AssertionError(f"layer table {seg_end} / {seg_k} was accepted")
+
+
+ALL_PINS = [pin_layered_bruteforce, pin_layered_special_cases, pin_layered_rejects_bad_tables, pin_tanh, pin_bruteforce_selector, pin_dense_passthrough, pin_reduces_to_topk,
             pin_error_feedback_identity, pin_toy_example, pin_table1_iteration1, pin_distortion_cases,
             pin_regularised_ranking, pin_aggregation, pin_pow, pin_exponent_variant, pin_model_update, pin_bf16_gradients, pin_select_modes_agree,
             pin_mask_certificate]

@@ -45,6 +45,12 @@ MUTANTS = [
     ("tanh_saturates_early", "if (x >= 9.25f) return 1.0f;", "if (x >= 2.0f) return 1.0f;"),
     ("bf16_shift", "static_cast<uint32_t>(h) << 16", "static_cast<uint32_t>(h) << 15"),
     ("nth_element_off_by_one", "rec.begin() + k, rec.end(), ranks_before);", "rec.begin() + k + 1, rec.end(), ranks_before);"),
+    ("layered_ignores_layer_start", "for (int64_t j = begin; j < end; ++j) rec.push_back", "for (int64_t j = 0; j < end; ++j) rec.push_back"),
+    ("layered_global_k", "for (int64_t i = 0; i < kl; ++i) chosen[i] = rec[i].idx;", "for (int64_t i = 0; i < kl; ++i) chosen[i] = rec[(i + 1) % rec.size()].idx;"),
+    ("layered_sends_score", "out_val[out] = a[j];   // the raw accumulator", "out_val[out] = score[j];   // the raw accumulator"),
+    ("layered_residual_not_cleared", "eps[j] = 0.0f;         // a - a", ";"),
+    ("layered_residual_not_carried", "eps[j] = a[j];  // (a minus 0", "eps[j] = 0.0f;  // (a minus 0"),
+    ("layered_accepts_gap", "if (begin != d) return -1;", ";"),
     ("certificate_strict", "if (!ranks_before(last, r)) ++count;", "if (ranks_before(r, last)) ++count;"),
 ]
 
