@@ -93,7 +93,7 @@ int regtopk_worker_step(regtopk_ctx* ctx, const void* grads, int64_t grad_ld, in
                         float* out_val);
 
 /* Accumulate-in-place form of the same round, for callers whose gradient computation can add into a
- * buffer (a backward pass that accumulates): Algorithm 2 step 6, a_n^t = eps_n^t + g_n^t, is then the
+ * buffer (a backward pass that accumulates): Algorithm 2 step 7, a_n^t = eps_n^t + g_n^t, is then the
  * caller's own addition, and the library never reads a separate gradient array nor rewrites the
  * accumulator: 4 bytes of memory traffic per coordinate and worker instead of 12.
  *   regtopk_accumulator gives the device pointer to the library's rows ([N][*ld] binary32, row n at
@@ -101,8 +101,8 @@ int regtopk_worker_step(regtopk_ctx* ctx, const void* grads, int64_t grad_ld, in
  *   regtopk_worker_step_inplace the caller, on the context's stream (or ordered before it), adds
  *   g_n^t[j] to element j of row n for j < d, in binary32 with a single round-to-nearest addition
  *   per element; elements [d, *ld) must stay 0.  The context's grad_dtype is not used by this form.
- *   regtopk_worker_step_inplace then does what regtopk_worker_step does from its accumulate step on
- *   (steps 7-12), with the same outputs, errors and call order; the two forms may be mixed from round
+ *   regtopk_worker_step_inplace then does what regtopk_worker_step does after its accumulate step
+ *   (steps 8-12), with the same outputs, errors and call order; the two forms may be mixed from round
  *   to round, and the results are bit-identical to regtopk_worker_step given the same gradients. */
 int regtopk_accumulator(regtopk_ctx* ctx, float** dev_ptr, int64_t* ld);
 int regtopk_worker_step_inplace(regtopk_ctx* ctx, int32_t* out_idx, float* out_val);
@@ -149,7 +149,9 @@ int regtopk_round_host(regtopk_ctx* ctx, const void* h_grads, int64_t grad_ld, i
                        float* h_val, float* h_g);
 
 /* Synchronises the stream and returns REGTOPK_OK or the sticky error recorded by the device
- * (REGTOPK_ERR_INTERNAL) or by CUDA (REGTOPK_ERR_CUDA). */
+ * (REGTOPK_ERR_INTERNAL) or by CUDA (REGTOPK_ERR_CUDA); a device error survives regtopk_state_reset.
+ * The checked build of the library (-DREGTOPK_DEBUG=1) also returns REGTOPK_ERR_INVALID_ARG here once an
+ * accumulator was infinite or NaN (gradients must be finite), until the next regtopk_state_reset. */
 int regtopk_status(regtopk_ctx* ctx);
 
 typedef struct {
@@ -184,7 +186,10 @@ int regtopk_debug_residual(regtopk_ctx* ctx, const float** dev_ptr, int64_t* ld)
  * the workers added in the order 0..N-1, but takes the pairs as arguments and keeps its scratch (one
  * bitmask row per worker) in a fixed array that is part of the library image instead of a workspace.
  *   idx, val  [N][k] pairs as regtopk_worker_step writes them: per worker distinct indices in
- *             ascending order.  omega: HOST array of N weights, or NULL for 1/N each.
+ *             ascending order.  The pairs are the caller's data and are not trusted: a pair whose index
+ *             lies outside [0, d) is ignored, and nothing outside the scratch rows and out_g is written
+ *             whatever the arrays hold (rows that are not ascending or repeat an index give an
+ *             unspecified but in-bounds result).  omega: HOST array of N weights, or NULL for 1/N each.
  *   out_g     [d] binary32, fully overwritten.
  * Limits: N <= REGTOPK_STATIC_MAX_WORKERS and N * ceil(d/32 rounded up to 4) <= REGTOPK_STATIC_SCRATCH_WORDS
  * (8 MiB of scratch, which every GPU that loads the library holds until the process exits); larger

@@ -39,6 +39,8 @@
 
 #include <cooperative_groups.h>
 #include <cuda_runtime.h>
+
+#include <atomic>
 #include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
@@ -89,8 +91,13 @@ enum : u32 { kErrCountMismatch = 1u, kErrDenseSelect = 2u, kErrRefine = 4u, kErr
 #if REGTOPK_DEBUG
 __device__ unsigned int g_bounds_faults;
 #define RT_INB(cond) ((cond) ? true : (atomicAdd(&g_bounds_faults, 1u), false))
+// Gradients must be finite.  The checked build counts the accumulators that are not (infinity or NaN) as the streaming
+// pass forms them; regtopk_status then reports REGTOPK_ERR_INVALID_ARG until regtopk_state_reset.
+__device__ unsigned int g_nonfinite;
+#define RT_NOTE_NONFINITE(key, in) do { if ((in) && (key) > 0x7F7FFFFFu) atomicAdd(&g_nonfinite, 1u); } while (0)
 #else
 #define RT_INB(cond) true
+#define RT_NOTE_NONFINITE(key, in) do { } while (0)
 #endif
 
 struct WorkerCtl {
@@ -433,7 +440,6 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
       ctl->bcount = 0;
       ctl->acount = 0;
       ctl->n_valid = 0;
-    ctl->b1 = kFull; ctl->above1 = 0; ctl->go_dense = 0; ctl->took_dense = 0;
       ctl->b1 = kFull; ctl->above1 = 0; ctl->go_dense = 0; ctl->took_dense = 0;
     }
     return;
@@ -779,6 +785,8 @@ __global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC, INPLACE
         }
         const u32 k0 = __float_as_uint(a.x) & 0x7FFFFFFFu, k1 = __float_as_uint(a.y) & 0x7FFFFFFFu;
         const u32 k2 = __float_as_uint(a.z) & 0x7FFFFFFFu, k3 = __float_as_uint(a.w) & 0x7FFFFFFFu;
+        RT_NOTE_NONFINITE(k0, full || j + 0 < p.d); RT_NOTE_NONFINITE(k1, full || j + 1 < p.d);
+        RT_NOTE_NONFINITE(k2, full || j + 2 < p.d); RT_NOTE_NONFINITE(k3, full || j + 3 < p.d);
         const bool h0 = k0 >= cutoff && (full || j + 0 < p.d);
         const bool h1 = k1 >= cutoff && (full || j + 1 < p.d);
         const bool h2 = k2 >= cutoff && (full || j + 2 < p.d);
@@ -1630,6 +1638,7 @@ static __device__ __align__(256) u32 g_static_scratch[REGTOPK_STATIC_SCRATCH_WOR
 
 struct StaticAggArgs {
   float* g;
+  int64_t d;
   int N;
   int64_t k;
   const int32_t* idx;
@@ -1639,13 +1648,24 @@ struct StaticAggArgs {
   float omega[REGTOPK_STATIC_MAX_WORKERS];
 };
 
+// The pairs come from the caller, not from the library's own selection, so every index is tested against
+// [0, d) before it addresses the scratch or g; a pair that fails is ignored (the checked build counts it).
+__device__ __forceinline__ bool static_index_ok(int32_t j, int64_t d) {
+  if ((u32)j < (u32)d) return true;
+#if REGTOPK_DEBUG
+  atomicAdd(&g_bounds_faults, 1u);
+#endif
+  return false;
+}
+
 __global__ void __launch_bounds__(256) k_static_mark(StaticAggArgs p) {
   const int64_t total = p.k * p.N;
   for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
        t += (int64_t)gridDim.x * blockDim.x) {
     const int n = (int)(t / p.k);
-    const u32 j = (u32)p.idx[t];
-    atomicOr(&p.mask[(size_t)n * p.W + (j >> 5)], 1u << (j & 31));
+    const int32_t j = p.idx[t];
+    if (!static_index_ok(j, p.d)) continue;
+    atomicOr(&p.mask[(size_t)n * p.W + ((u32)j >> 5)], 1u << (j & 31));
   }
 }
 
@@ -1658,6 +1678,7 @@ __global__ void __launch_bounds__(256) k_static_aggregate(StaticAggArgs p) {
        t += (int64_t)gridDim.x * blockDim.x) {
     const int n = (int)(t / p.k);
     const int32_t j = p.idx[t];
+    if (!static_index_ok(j, p.d)) continue;
     const size_t wi = (size_t)((u32)j >> 5);
     const u32 bm = 1u << (j & 31);
     bool owned = true;
@@ -1672,7 +1693,8 @@ __global__ void __launch_bounds__(256) k_static_aggregate(StaticAggArgs p) {
         const int64_t mid = (lo + hi) >> 1;
         if (row[mid] < j) lo = mid + 1; else hi = mid;
       }
-      sum = __fadd_rn(sum, __fmul_rn(p.omega[m], p.val[(size_t)m * p.k + lo]));
+      // rows that are not ascending can send the search past the entry: such a term is left out
+      if (lo < p.k && row[lo] == j) sum = __fadd_rn(sum, __fmul_rn(p.omega[m], p.val[(size_t)m * p.k + lo]));
     }
     sum = __fadd_rn(sum, __fmul_rn(p.omega[n], p.val[t]));
     p.g[j] = sum;
@@ -1893,6 +1915,21 @@ size_t regtopk_workspace_bytes(int64_t d, int32_t N, int64_t k, const regtopk_pa
 
 int regtopk_state_reset(regtopk_ctx* c) {
   if (!c) return REGTOPK_ERR_INVALID_ARG;
+  // The device's error word lives in the memory cleared below: an error it holds becomes the context's sticky
+  // code first, so that a reset cannot lose it (this read synchronises the stream; resets are rare).
+  if (c->round > 0 || c->stepped) {
+    GlobalCtl h;
+    memset(&h, 0, sizeof h);
+    if (cudaMemcpyAsync(&h, c->ws + c->L.off_gctl, sizeof h, cudaMemcpyDeviceToHost, c->stream) == cudaSuccess &&
+        cudaStreamSynchronize(c->stream) == cudaSuccess && h.err && !c->sticky)
+      c->sticky = REGTOPK_ERR_INTERNAL;
+  }
+#if REGTOPK_DEBUG
+  {
+    const unsigned int zero = 0;
+    cudaMemcpyToSymbolAsync(g_nonfinite, &zero, sizeof zero, 0, cudaMemcpyHostToDevice, c->stream);
+  }
+#endif
   int rc = note_cuda(c, cudaMemsetAsync(c->ws, 0, c->L.zero_end, c->stream));
   c->round = 0;
   c->stepped = 0;
@@ -2240,6 +2277,9 @@ int regtopk_status(regtopk_ctx* c) {
   unsigned int faults = 0;
   if (cudaMemcpyFromSymbol(&faults, g_bounds_faults, sizeof faults) != cudaSuccess) return note_cuda(c, cudaErrorUnknown);
   if (faults) return REGTOPK_ERR_INTERNAL;
+  unsigned int nonfinite = 0;
+  if (cudaMemcpyFromSymbol(&nonfinite, g_nonfinite, sizeof nonfinite) != cudaSuccess) return note_cuda(c, cudaErrorUnknown);
+  if (!h.err && nonfinite) return REGTOPK_ERR_INVALID_ARG;
 #endif
   return h.err ? REGTOPK_ERR_INTERNAL : REGTOPK_OK;
 }
@@ -2316,21 +2356,24 @@ int regtopk_aggregate_pairs_static(int64_t d, int32_t N, int64_t k, const int32_
   if (N > REGTOPK_STATIC_MAX_WORKERS) return REGTOPK_ERR_TOO_LARGE;
   const int64_t W = ((d + 31) / 32 + 3) / 4 * 4;
   if ((int64_t)N * W > (int64_t)REGTOPK_STATIC_SCRATCH_WORDS) return REGTOPK_ERR_TOO_LARGE;
-  // Device address of the scratch array, looked up once per device with that device current.
-  static u32* scratch_of_device[64] = {nullptr};
+  // Device address of the scratch array, looked up once per device with that device current.  The cache is
+  // written with release and read with acquire order: threads that race here all store the same address.
+  static std::atomic<u32*> scratch_of_device[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return REGTOPK_ERR_NO_DEVICE;
-  if (!scratch_of_device[dev]) {
+  u32* scratch = scratch_of_device[dev].load(std::memory_order_acquire);
+  if (!scratch) {
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
       cudaGetLastError();
       return REGTOPK_ERR_NO_DEVICE;
     }
-    scratch_of_device[dev] = static_cast<u32*>(ptr);
+    scratch = static_cast<u32*>(ptr);
+    scratch_of_device[dev].store(scratch, std::memory_order_release);
   }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   StaticAggArgs a;
-  a.g = out_g; a.N = N; a.k = k; a.idx = idx; a.val = val; a.mask = scratch_of_device[dev]; a.W = W;
+  a.g = out_g; a.d = d; a.N = N; a.k = k; a.idx = idx; a.val = val; a.mask = scratch; a.W = W;
   for (int n = 0; n < REGTOPK_STATIC_MAX_WORKERS; ++n) {
     a.omega[n] = n < N ? (omega ? omega[n] : 1.0f / (float)N) : 0.0f;
     if (n < N && !isfinite(a.omega[n])) return REGTOPK_ERR_INVALID_ARG;

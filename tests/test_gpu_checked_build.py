@@ -36,6 +36,22 @@ for name in ("resnet18", "gpt2"):
     for k in w.k_values():
         s = synth.GradientStream(w, device="cpu", seed=17, pad_to=8)
         stats.append(run_parity((s.next() for _ in range(6)), w.d, w.N, max(k, 1), w.mu))
+# non-finite gradients: the checked build says so through status(), and a reset clears it
+from paper_2501_05633_b200 import RegTopK
+from paper_2501_05633_b200.binding import RegTopKError
+lib = RegTopK(50_000, 2, 500)
+g = torch.randn(2, 50_000)
+lib.worker_step(g.cuda()); lib.aggregate(); lib.status()
+g[1, 77] = float("inf")
+lib.worker_step(g.cuda()); lib.aggregate()
+try:
+    lib.status()
+    raise SystemExit("non-finite accumulator not reported")
+except RegTopKError as e:
+    assert e.code == -1, e.code
+lib.state_reset()
+lib.worker_step(torch.randn(2, 50_000).cuda()); lib.aggregate(); lib.status()
+lib.close()
 bad = [st for st in stats if st["device_error_bits"]]
 assert not bad, bad
 assert binding.library_path().endswith("libregtopk_checked.so")

@@ -382,37 +382,77 @@ def test_fused_model_update_trajectory():
 
 
 def test_state_export_import_resumes_bit_identically():
+    """A context restored from an exported blob continues exactly as the oracle does (which ran all rounds without
+    interruption), and so does the context that exported."""
+    from oracle.oracle import OracleRegTopK
     d, N, k = 150_001, 3, 1500
-    rounds = [x.cuda() for x in gauss_rounds(N, d, 7, seed=91)]
+    rounds = list(gauss_rounds(N, d, 7, seed=91))
+    ora = OracleRegTopK(d, N, k, 4.0)
+    want = []
+    for g in rounds:
+        oi, ov = ora.worker_step(g.numpy())
+        want.append((oi, ov.view(np.uint32).copy(), ora.eps.view(np.uint32).copy(), ora.aggregate().view(np.uint32).copy()))
+
+    def check(lib, t):
+        idx, val = lib.worker_step(rounds[t].cuda())
+        eps = lib.residual().cpu().numpy().view(np.uint32)
+        agg = lib.aggregate().cpu().numpy().view(np.uint32)
+        oi, ov, oe, og = want[t]
+        assert np.array_equal(idx.cpu().numpy(), oi), f"round {t}: index sets"
+        assert np.array_equal(val.cpu().numpy().view(np.uint32), ov), f"round {t}: values"
+        assert np.array_equal(eps, oe), f"round {t}: residuals"
+        assert np.array_equal(agg, og), f"round {t}: aggregate"
+
     a = RegTopK(d, N, k)
-    for g in rounds[:4]:
-        a.worker_step(g)
-        a.aggregate()
+    for t in range(4):
+        check(a, t)
     blob = a.state_export()
-    a.worker_step(rounds[4])
+    a.worker_step(rounds[4].cuda())
     with pytest.raises(RegTopKError) as e:  # mid-round: refused
         a.state_export()
     assert e.value.code == -3
     a.aggregate()
-    ref = []
-    for g in rounds[5:]:
-        idx, val = a.worker_step(g)
-        ref.append((idx.clone(), val.clone(), a.aggregate().clone(), a.residual().clone()))
+    for t in (5, 6):
+        check(a, t)
     b = RegTopK(d, N, k)
     b.state_import(blob)
-    b.worker_step(rounds[4])
-    b.aggregate()
-    for g, want in zip(rounds[5:], ref):
-        idx, val = b.worker_step(g)
-        got = (idx, val, b.aggregate(), b.residual())
-        for x, y in zip(got, want):
-            assert torch.equal(x, y)
+    for t in (4, 5, 6):
+        check(b, t)
     b.status()
     other = RegTopK(d, N, k + 1)
     with pytest.raises(RegTopKError):  # a blob of a different problem
         other.state_import(blob)
     with pytest.raises(RegTopKError):
         b.state_import(blob[:1000].clone())
+
+
+def test_appendix_a_table1_iteration1_on_the_library():
+    """The low-dimensional example of Appendix A (J = 4, two workers, Top-3 / RegTop-3, omega = 1/2): the accumulated
+    gradients reconstructed from Table 1's iteration-1 row go through the C ABI; each worker drops the entry the table
+    shows as dropped, the sent values are the printed ones, and the aggregate is the printed target without the dropped
+    entries' share.  Bit-identical to the oracle as well."""
+    import json
+    import os
+    from oracle.oracle import OracleRegTopK
+    fx = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "table1_iteration1.json")))
+    acc = np.array(fx["worker_accumulated"], np.float32)
+    sent = np.array(fx["worker_sent"], np.float64)
+    for mu in (0.0, 4.0):  # iteration 1 has no previous mask: the same for Top-k and RegTop-k
+        lib = RegTopK(4, 2, 3, mu=mu, omega=[0.5, 0.5])
+        ora = OracleRegTopK(4, 2, 3, mu, omega=[0.5, 0.5])
+        idx, val = lib.worker_step(torch.from_numpy(acc).cuda())
+        g = lib.aggregate().cpu().numpy()
+        lib.status()
+        idx_h, val_h = idx.cpu().numpy(), val.cpu().numpy()
+        for n in range(2):
+            dense = np.zeros(4)
+            dense[idx_h[n]] = val_h[n]
+            assert np.allclose(dense, sent[n], atol=0.006)
+            assert set(range(4)) - set(int(i) for i in idx_h[n]) == {fx["dropped_index_0based"][n]}
+        assert np.allclose(g, sent.mean(axis=0), atol=0.006)
+        oi, ov = ora.worker_step(acc)
+        assert np.array_equal(idx_h, oi) and np.array_equal(val_h.view(np.uint32), ov.view(np.uint32))
+        assert np.array_equal(g.view(np.uint32), ora.aggregate().view(np.uint32))
 
 
 # ---- API behaviour -------------------------------------------------------------------------------------------
@@ -549,7 +589,8 @@ def _certified_round(lib, ora_api, w, k, grads, eps_before, prev, g_prev, omega)
     return (idx_h, val_h), agg
 
 
-@pytest.mark.parametrize("name,ki,rounds", [("gpt2", 0, 2), ("gpt2", 1, 2), ("flat1p3b", 1, 2)])
+@pytest.mark.parametrize("name,ki,rounds", [("gpt2", 0, 2), ("gpt2", 1, 2), ("flat1p3b", 0, 2), ("flat1p3b", 1, 2),
+                                            ("flat1p3b", 2, 2)])
 def test_full_size_certified(name, ki, rounds):
     import psutil
     from oracle.oracle import default as oracle_default
