@@ -52,6 +52,9 @@ def parse():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--select", default="global", choices=["global", "layerwise", "dense"],
+                    help="layerwise: every tensor of the workload keeps its own share (one Top-k per layer); dense: the "
+                         "exact full-grid selection from the rows is forced every round (the path a missed cutoff takes)")
     ap.add_argument("--api", default="plain", choices=["plain", "inplace"],
                     help="inplace: the step is the caller's accumulate (torch add_ into the library's rows) + "
                          "regtopk_worker_step_inplace + regtopk_aggregate; the library's share is reported beside it")
@@ -235,14 +238,28 @@ class Bench:
         self.ring = None
         self.torch.cuda.empty_cache()
 
-    def variant(self, ki, steps, warmup, api="plain", flags=0, per_step_events=False, sampler=None, barrier=None):
+    def layers(self, ki):
+        """Every tensor of the workload as a layer that keeps the workload's share of its entries (at least one)."""
+        import itertools
+        frac = self.w.sparsity[ki]
+        ends = list(itertools.accumulate(self.w.shapes))
+        ks = [int(min(n, max(1, int(frac * n + 0.5)))) for n in self.w.shapes]
+        return ends, ks
+
+    def variant(self, ki, steps, warmup, api="plain", flags=0, per_step_events=False, sampler=None, barrier=None,
+                select="global"):
         """Times `steps` rounds after `warmup` (at least 3) with CUDA events on the library's stream (torch's current
         stream); then the same rounds again with an event pair around the streaming kernel.  Returns a dict."""
         torch = self.torch
         import paper_2501_05633_b200 as pkg
         w, ring, ring_n = self.w, self.ring, self.ring_n
         k = w.k_values()[ki]
-        lib = pkg.RegTopK(w.d, w.N, k, mu=w.mu, grad_dtype=self.tdt, flags=flags)
+        layers = self.layers(ki) if select == "layerwise" else None
+        if layers is not None:
+            k = int(sum(layers[1]))
+        if select == "dense":
+            flags |= binding_flags("dense")
+        lib = pkg.RegTopK(w.d, w.N, k, mu=w.mu, grad_dtype=self.tdt, flags=flags, layers=layers)
         out_idx = torch.empty((w.N, k), dtype=torch.int32, device=self.dev)
         out_val = torch.empty((w.N, k), dtype=torch.float32, device=self.dev)
         inplace = api == "inplace"
@@ -316,12 +333,17 @@ class Bench:
                 "candidates_last": stats_end["candidates_last"], "step": step}
 
 
-def sweep_entry(b, r, ki, api, peak):
+def binding_flags(select):
+    from paper_2501_05633_b200 import binding
+    return (binding.FLAG_FORCE_DENSE_SELECT | binding.FLAG_GRID_DENSE_SELECT) if select == "dense" else 0
+
+
+def sweep_entry(b, r, ki, api, peak, select="global"):
     w = b.w
     ms_step = r["ms_total"] / r["steps"]
     step_gbs = r["alg_bytes"] / (ms_step * 1e-3) / 1e9
     kern_gbs = r["kern_alg_bytes"] / (r["kern_avg_ms"] * 1e-3) / 1e9 if r["kern_avg_ms"] > 0 else None
-    e = {"workload": workload_label(w, r["k"], w.sparsity[ki]), "api": api, "steps": r["steps"], "ms_per_step": ms_step,
+    e = {"workload": workload_label(w, r["k"], w.sparsity[ki]), "api": api, "select": select, "steps": r["steps"], "ms_per_step": ms_step,
          "g_coords_per_s": r["coords"] / (ms_step * 1e-3) / 1e9, "step_hbm_gbs": step_gbs,
          "step_frac_of_8TBs": step_gbs / 8000.0, "step_frac_of_measured_peak": step_gbs / peak,
          "k_stream_ms": r["kern_avg_ms"], "k_stream_gbs": kern_gbs,
@@ -391,6 +413,13 @@ def main():
                 r["lib"].close()
                 del r
                 torch.cuda.empty_cache()
+            if name in ("resnet18", "gpt2"):  # layer-wise selection, and the forced dense exact path, on two shapes
+                for sel in ("layerwise", "dense"):
+                    r = b.variant(0, max(10, n_steps // 4), args.warmup, select=sel)
+                    sweep.append(sweep_entry(b, r, 0, "plain", peak, select=sel))
+                    r["lib"].close()
+                    del r
+                    torch.cuda.empty_cache()
             if name != head_name:
                 b.close()
                 del b
@@ -403,7 +432,7 @@ def main():
     sampler = ClockSampler(local) if rank == 0 else None
     flags = binding.FLAG_HOST_STAGING if (args.e2e_steps > 0 and args.api == "plain") else 0
     r = head.variant(head_ki, args.steps, args.warmup, api=args.api, flags=flags, per_step_events=True,
-                     sampler=sampler, barrier=barrier)
+                     sampler=sampler, barrier=barrier, select=args.select)
     lib, k, step = r["lib"], r["k"], r["step"]
     inplace = args.api == "inplace"
     # round 0 (no previous support: Algorithm 1) on its own
@@ -450,7 +479,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": w.grad_dtype, "data": "synthetic",
             "config": {"workload": workload_label(w, k, w.sparsity[head_ki]),
-                       "replicas": world, "parallelism": "replicas only (one context runs on one GPU)",
+                       "select": args.select, "replicas": world, "parallelism": "replicas only (one context runs on one GPU)",
                        "l2": f"inputs larger than L2 ({head.per_batch / 1e6:.0f} MB per step, ring of {head.ring_n} batches)",
                        "step_hbm_gbs": step_gbs, "step_frac_of_measured_peak": step_gbs / peak,
                        "step_frac_of_8TBs": step_gbs / 8000.0,

@@ -52,8 +52,10 @@ enum { REGTOPK_GRAD_F32 = 0, REGTOPK_GRAD_BF16 = 1 };
 enum {
   REGTOPK_FLAG_HOST_STAGING = 1,      /* reserve workspace for regtopk_round_host                          */
   REGTOPK_FLAG_FORCE_DENSE_SELECT = 2, /* testing: skip the sampled cutoff, always take the dense exact path */
-  REGTOPK_FLAG_FORCE_WIDE_LISTS = 4    /* testing: handle the candidate lists the way large N*k is handled (separate
+  REGTOPK_FLAG_FORCE_WIDE_LISTS = 4,   /* testing: handle the candidate lists the way large N*k is handled (separate
                                           full-grid kernels, pairs unzipped afterwards) at any size; same results */
+  REGTOPK_FLAG_GRID_DENSE_SELECT = 8   /* testing: when a worker needs the dense exact path, run it as the full-grid
+                                          kernel that large problems use, at any size; same results              */
 };
 
 typedef struct {
@@ -64,6 +66,17 @@ typedef struct {
   float y;             /* exponent of Remark 3: selection metric |a|^y * regulariser, 0 < y <= 1; 0 or 1 means
                           Algorithm 2 as printed.  The mask is computed by ranking |a| * regulariser^(1/y), which
                           orders the entries the same way.                                                   */
+  /* Layer-wise sparsification (one Top-k per layer instead of one over the whole vector; the paper's
+     related-work section cites it).  n_layers == 0: Algorithm 2 as printed, one selection over all d
+     coordinates.  n_layers >= 1: layer l is the contiguous index range [layer_end[l-1], layer_end[l])
+     (layer_end ascending, layer_end[n_layers-1] == d) and keeps its layer_k[l] largest scores
+     (1 <= layer_k[l] <= the layer's size); the k given to regtopk_create must equal the sum of layer_k.
+     Accumulator, distortion, regulariser, sent values, residual and aggregation are unchanged; a worker's
+     k pairs still come out in ascending index order.  Both arrays are host memory, read during
+     regtopk_workspace_bytes and regtopk_create only.                                                     */
+  int32_t n_layers;
+  const int64_t* layer_end;
+  const int64_t* layer_k;
 } regtopk_params;
 
 /* Bytes of device workspace a context for (d, N, k) needs; 0 if the arguments are invalid.

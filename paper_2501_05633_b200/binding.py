@@ -20,7 +20,7 @@ _LIB = os.path.join(_PKG, "libregtopk.so")
 
 OK = 0
 GRAD_F32, GRAD_BF16 = 0, 1
-FLAG_HOST_STAGING, FLAG_FORCE_DENSE_SELECT, FLAG_FORCE_WIDE_LISTS = 1, 2, 4
+FLAG_HOST_STAGING, FLAG_FORCE_DENSE_SELECT, FLAG_FORCE_WIDE_LISTS, FLAG_GRID_DENSE_SELECT = 1, 2, 4, 8
 
 EXPORTS = [
     "regtopk_workspace_bytes", "regtopk_create", "regtopk_worker_step", "regtopk_aggregate",
@@ -33,7 +33,9 @@ EXPORTS = [
 
 class Params(ctypes.Structure):
     _fields_ = [("mu", ctypes.c_float), ("omega", ctypes.POINTER(ctypes.c_float)),
-                ("grad_dtype", ctypes.c_int32), ("flags", ctypes.c_int32), ("y", ctypes.c_float)]
+                ("grad_dtype", ctypes.c_int32), ("flags", ctypes.c_int32), ("y", ctypes.c_float),
+                ("n_layers", ctypes.c_int32), ("layer_end", ctypes.POINTER(ctypes.c_int64)),
+                ("layer_k", ctypes.POINTER(ctypes.c_int64))]
 
 
 class Stats(ctypes.Structure):
@@ -145,16 +147,28 @@ def _check(code: int, where: str):
         raise RegTopKError(code, where)
 
 
-def _make_params(mu, omega, grad_dtype, flags, y=1.0):
+def _make_params(mu, omega, grad_dtype, flags, y=1.0, layers=None):
+    """layers: None, or (layer_end, layer_k), two equally long integer sequences (see regtopk_params)."""
     p = Params()
     p.mu = float(mu)
-    keep = None
+    keep = []
     if omega is not None:
-        keep = (ctypes.c_float * len(omega))(*[float(x) for x in omega])
-        p.omega = ctypes.cast(keep, ctypes.POINTER(ctypes.c_float))
+        om = (ctypes.c_float * len(omega))(*[float(x) for x in omega])
+        keep.append(om)
+        p.omega = ctypes.cast(om, ctypes.POINTER(ctypes.c_float))
     p.grad_dtype = grad_dtype
     p.flags = flags
     p.y = float(y)
+    if layers is not None:
+        ends, ks = [int(x) for x in layers[0]], [int(x) for x in layers[1]]
+        if len(ends) != len(ks) or not ends:
+            raise ValueError("layers = (layer_end, layer_k) of equal, non-zero length")
+        e = (ctypes.c_int64 * len(ends))(*ends)
+        kk = (ctypes.c_int64 * len(ks))(*ks)
+        keep += [e, kk]
+        p.n_layers = len(ends)
+        p.layer_end = ctypes.cast(e, ctypes.POINTER(ctypes.c_int64))
+        p.layer_k = ctypes.cast(kk, ctypes.POINTER(ctypes.c_int64))
     return p, keep
 
 
@@ -185,8 +199,8 @@ def aggregate_pairs_static(idx: torch.Tensor, val: torch.Tensor, d: int, omega=N
     return out
 
 
-def workspace_bytes(d, N, k, mu=4.0, omega=None, grad_dtype=GRAD_F32, flags=0, y=1.0) -> int:
-    p, _keep = _make_params(mu, omega, grad_dtype, flags, y)
+def workspace_bytes(d, N, k, mu=4.0, omega=None, grad_dtype=GRAD_F32, flags=0, y=1.0, layers=None) -> int:
+    p, _keep = _make_params(mu, omega, grad_dtype, flags, y, layers)
     return int(load_library().regtopk_workspace_bytes(d, N, k, ctypes.byref(p)))
 
 
@@ -194,13 +208,15 @@ class RegTopK:
     """One (d, N, k) sparsifier context on the current CUDA device.
 
     grads: torch tensor [N, ld] on the device, float32 or bfloat16 as chosen at construction.
+    layers = (layer_end, layer_k) selects layer by layer (regtopk_params.n_layers); k is then their sum.
     worker_step returns (idx [N,k] int32, val [N,k] float32); aggregate returns g [d] float32 (a view of
     the library's state unless `out` is given).  Work is enqueued on `stream` (default: torch's current
     stream at construction) and is asynchronous like any torch CUDA op.
     """
 
     def __init__(self, d: int, N: int, k: int, mu: float = 4.0, omega=None, grad_dtype=torch.float32,
-                 flags: int = 0, device=None, stream: Optional[torch.cuda.Stream] = None, y: float = 1.0):
+                 flags: int = 0, device=None, stream: Optional[torch.cuda.Stream] = None, y: float = 1.0,
+                 layers=None):
         if not torch.cuda.is_available():
             raise RuntimeError("RegTopK needs a CUDA device; there is no CPU implementation")
         self.L = load_library()
@@ -212,7 +228,10 @@ class RegTopK:
             raise TypeError("gradients are float32 or bfloat16")
         self.flags = int(flags)
         self.y = float(y)
-        p, keep = _make_params(mu, omega, self.dtype_code, self.flags, self.y)
+        if layers is not None:  # layer-wise selection: k is the sum of the per-layer k
+            k = int(sum(int(x) for x in layers[1]))
+            self.k = k
+        p, keep = _make_params(mu, omega, self.dtype_code, self.flags, self.y, layers)
         nbytes = int(self.L.regtopk_workspace_bytes(self.d, self.N, self.k, ctypes.byref(p)))
         if nbytes == 0:
             raise RegTopKError(-1, "regtopk_workspace_bytes")

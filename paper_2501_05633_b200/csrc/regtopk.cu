@@ -116,12 +116,13 @@ struct WorkerCtl {
                     // selection had to fall back to the dense path, counted down by k_sample_cutoff, and kept
                     // across rounds (nothing else resets it but regtopk_state_reset)
   u32 exact_window; // length of the last such stretch: it doubles with every further fallback
-  u32 pad[3];
+  u32 hint;         // the sampled cutoff of this round, kept for k_dense when the candidate path is not taken (0xFFFFFFFF: none)
+  u32 pad[2];
 };
 
 struct GlobalCtl {
   u32 err;
-  u32 pad;
+  u32 dense_flags;    // k_dense: kFlag* bits that all blocks of the launch read after a grid barrier; zero between launches
   u64 dense_workers;
 };
 
@@ -329,7 +330,7 @@ struct SampleArgs {
   u32* ghist;  // [N][4][kBins] histograms of k_post, cleared here
   u32* shist;  // [N][kSampleBins] histogram of this kernel; zero on entry (k_post clears it again)
   u32* skeys;  // [N][kSampleMax] the sample's keys (0xFFFFFFFF in unused slots), for the exact second look
-  int force_dense;
+  int force_dense;  // 1: no sampling, the dense path is taken; 2: sample, keep the cutoff as a hint, take the dense path
   // Clusters beyond the first N compute the regularised scores of the previous support
   // (Eq. (Delta_def), Algorithm 2 steps 8-9) while the first N sample.  On that support the
   // residual is +0, so the accumulator there is 0 + g.
@@ -431,8 +432,9 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
 
   for (int i = rk * blockDim.x + tid; i < 4 * kBins; i += kSampleCluster * blockDim.x)
     p.ghist[(size_t)n * 4 * kBins + i] = 0;
-  if (p.force_dense) {  // the same in every block: nobody reaches a barrier
+  if (p.force_dense == 1) {  // the same in every block: nobody reaches a barrier
     if (rk == 0 && tid == 0) {
+      ctl->hint = kFull;
       ctl->cutoff = kFull;  // no key reaches it: the stream pass collects nothing
       ctl->bin_shift = 0;
       ctl->cand_count = 0;
@@ -571,10 +573,12 @@ __global__ void __launch_bounds__(kBlockSel) k_sample_cutoff(SampleArgs p) {
     u32 shift = 0;
     while ((range >> shift) > (u32)(kBins - 2)) ++shift;
     if (want_exact) ctl->exact_rounds -= 1u;
-    ctl->cutoff = cutoff;
+    ctl->hint = cutoff;
+    // force_dense == 2: the dense path is asked for, on the whole grid; the cutoff only serves it as a hint
+    ctl->cutoff = p.force_dense == 2 ? kFull : cutoff;
     ctl->bin_shift = shift;
     ctl->cand_count = 0;
-    ctl->force_dense = 0;
+    ctl->force_dense = p.force_dense == 2 ? 1u : 0u;
     ctl->bcount = 0;
     ctl->acount = 0;
     ctl->n_valid = 0;
@@ -865,6 +869,7 @@ struct PostArgs {
   int has_stale;  // mask_new holds an old mask (round >= 2)
   int pair_mode;  // many pairs: emit (index, value) as one store into the B list; k_unzip follows
   int wide;       // k_post runs between the wide kernels: refinement or dense path only
+  int grid_dense; // a worker that needs the dense exact path is left to k_dense (ctl->go_dense) instead of this cluster
 };
 
 __device__ __forceinline__ u32 warp_reserve_global(bool pred, u32* counter) {
@@ -1232,6 +1237,13 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
       cl.sync();  // (2) refinement list complete
     }
   }
+  if (dense && p.grid_dense) {  // the same in every block: k_dense, the next kernel, selects for this worker
+    if (rk == 0 && tid == 0) {
+      ctl->go_dense = 1u;
+      atomicAdd(&p.gctl->dense_workers, 1ull);
+    }
+    return;
+  }
 
   if (!dense) {
     const u32 nB = __ldcg(&ctl->bcount);
@@ -1523,6 +1535,802 @@ __global__ void __launch_bounds__(256) k_unzip(UnzipArgs p) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// k_dense: exact selection straight from the rows, by the whole grid (a cooperative launch; the phases are
+// separated by grid-wide barriers).  It serves the workers whose candidate path gave up (ctl->go_dense:
+// cutoff guessed too high, list overflowed, or the dense path was asked for) and every worker in
+// layer-wise mode, where each layer of a row is a selection problem of its own: a row is a sequence of
+// segments (one for the whole row in the plain mode), segment s keeps its k_s largest (score, lowest index).
+//
+// Per segment:
+//   (A) a histogram of the top 12 key bits over the segment's part of the row, restricted to keys at or above
+//       a lower bound `lo` (a hint: the sampled cutoff, or last round's threshold lowered by an octave), so
+//       that nearly all entries cost a compare and no shared-memory atomic.  From the top down, the bin b0 that
+//       holds the k_s-th largest, the entries above it and the number c0 inside it.  If the histogram holds
+//       fewer than k_s entries the hint was too high and the pass is repeated for that segment with lo = 0.
+//   (B) a second pass over the rows: entries above bin b0 are winners (mask bit set, composite appended to
+//       the worker's winner list); the c0 entries inside it go to a list of their own,
+//   (C) from which one block takes the `need` largest composites (key, lowest index).
+// A segment whose bin b0 does not fit the list space (rows full of equal values) stays on the rows instead:
+// two more digits of 12 and 7 bits give the threshold key T and the number of entries equal to T that are
+// to be taken; if there are more of those than needed, their counts per tile are scanned so that the lowest
+// indices win; a last pass over the rows sets the winners.
+// Rows are cut into tiles of kDenseTile coordinates that never straddle a segment; a block owns a
+// contiguous run of tiles.  If nobody needs the path the kernel returns at once.
+// ---------------------------------------------------------------------------------------------
+constexpr int kDenseThreads = 512;
+constexpr int kDenseUnroll = 4;   // quads a thread has in flight: 64 bytes, 64 KB per SM with two blocks of 512 threads
+constexpr int kDenseTile = kDenseUnroll * 4 * kDenseThreads;  // 8192 coordinates: one step of the walk
+constexpr int kDenseWarps = kDenseThreads / 32;
+constexpr int kDenseMaxFlagged = 1024;
+constexpr u32 kOctave = 0x00800000u;  // one binary order of magnitude in key units
+constexpr u32 kHintMargin = 2u << 19;  // two bins of the first digit (an eighth of an octave)
+
+enum : u32 { kSegList = 0u, kSegRows = 1u, kSegRetry = 2u };
+enum : u32 { kFlagRetry = 1u, kFlagRows = 2u, kFlagOrdered = 4u, kFlagBad = 8u };
+
+struct __align__(16) SegState {
+  u32 prefix;  // digits of the threshold key fixed so far
+  u32 need;    // entries still to be taken among those that match the prefix
+  u32 ties;    // entries in the bin of the last digit found (after the last digit: entries equal to the threshold key)
+  u32 mode;    // kSegList, kSegRows, or kSegRetry while the first digit has to be counted again
+  u32 lo;      // keys below this are left out of the first histogram
+  u32 boff;    // kSegList: where the segment's in-bin list starts in the worker's B list
+  u32 bfill;   //           entries written there so far
+  u32 pad;
+};
+
+struct DenseArgs {
+  PostArgs p;
+  int N;
+  int n_seg;
+  int finish;               // also rank the winners and emit the pairs (otherwise k_wide_prefix / k_wide_emit follow)
+  int layered;              // hints come from last round's thresholds (seg_thr), not from the sampled cutoff
+  u32 emit_segments;        // mask-row segments the emission and k_aggregate use
+  int64_t tiles;            // tiles per worker
+  const int64_t* seg_end;   // [n_seg] end of each segment (ascending, the last is d)
+  const int64_t* seg_kpre;  // [n_seg + 1] exclusive prefix sums of the segments' k
+  const int64_t* seg_tile0; // [n_seg + 1] first tile of each segment
+  u32* dhist;               // [N][n_seg][kBins], all zero between launches
+  SegState* seg;            // [N][n_seg]
+  u32* seg_thr;             // [N][n_seg] a lower bound of the segment's threshold key in the last round it came here (0: none)
+  u32* tile_ties;           // [N][tiles][2]: entries equal to the threshold key in the tile, and in lower tiles of the segment
+};
+
+__device__ __forceinline__ int dense_seg_of_tile(const int64_t* seg_tile0, int n_seg, int64_t t) {
+  int lo = 0, hi = n_seg;  // the last segment whose first tile is at or before t
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (seg_tile0[mid] <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// Calls f(j4, key, in) with the score keys of the quad j4 .. j4 + 3 (in[q]: the entry lies in [t0, t1)) for the
+// quads that meet [t0, t1), but only where some lane of the warp holds a key of at least min_key in its quad: the
+// call is made by all lanes of such a warp or by none, so f may use warp-wide primitives, and with min_key == 0 it
+// is made by every thread of the block the same number of times, so f may then use block-wide ones.  With
+// PER_THREAD only the threads whose own quad holds such a key call f (which must then do without warp-wide
+// primitives), and every lane calls after() once per step of the loop (kDenseUnroll quads), converged.  A thread's
+// quads within one step of the loop are 4 * blockDim.x coordinates apart, and threads hold consecutive quads.
+// kDenseUnroll 16-byte loads per thread are in flight.  Keys as in dense_key: the regularised score on the previous
+// support, bits(|a|) elsewhere.  With SKIP_MARKED the walk does not look at the previous support at all (no mask
+// word per quad, no binary search for a score: a chain of dependent loads that stalls the warp): every key is
+// bits(|a|); the caller sorts the previous support out afterwards (entries staged for a list are tested against
+// the old mask in batches when the list is written out; a histogram is corrected from the override list, which
+// holds those entries' scores in index order).
+struct NoHook { __device__ __forceinline__ void operator()() const {} };
+
+template <bool SKIP_MARKED, bool PER_THREAD = false, typename F, typename G = NoHook>
+__device__ __forceinline__ void dense_walk(const PostArgs& p, int n, int64_t t0, int64_t t1, u32 min_key, F f, G after = G()) {
+  const float* row = p.eps + (size_t)n * p.ld;
+  const u32* marks = (p.use_marks && !SKIP_MARKED) ? p.mask_old + (size_t)n * p.W : nullptr;
+  constexpr int kU = kDenseUnroll;
+  const int stride = 4 * (int)blockDim.x;
+  for (int64_t base = t0 & ~(int64_t)3; base < t1; base += kU * stride) {
+    // this step's part of [t0, t1) as offsets from base
+    const int lo_off = (int)(t0 - base);  // <= 3; negative after the first step
+    const int hi_off = t1 - base < (int64_t)kU * stride ? (int)(t1 - base) : kU * stride;
+    float4 e[kU];
+    u32 w[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const int off = u * stride + 4 * (int)threadIdx.x;
+      const bool live = off < hi_off;  // rows are padded to a multiple of 1024: the whole quad is inside the row's storage
+      e[u] = live ? __ldcs(reinterpret_cast<const float4*>(row + base + off)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      w[u] = (live && marks) ? (__ldg(marks + ((base + off) >> 5)) >> ((base + off) & 31)) & 15u : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      if (u * stride >= hi_off) break;  // the same in every thread
+      const int off = u * stride + 4 * (int)threadIdx.x;
+      const int64_t j4 = base + off;
+      u32 key[4] = {__float_as_uint(e[u].x) & 0x7FFFFFFFu, __float_as_uint(e[u].y) & 0x7FFFFFFFu,
+                    __float_as_uint(e[u].z) & 0x7FFFFFFFu, __float_as_uint(e[u].w) & 0x7FFFFFFFu};
+      bool in[4] = {true, true, true, true};
+      if (w[u] != 0u || off < lo_off || off + 4 > hi_off) {  // rare: an entry of the previous support, or a quad across an end
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          in[q] = off + q >= lo_off && off + q < hi_off;
+          if (!in[q]) key[q] = 0u;
+          else if ((w[u] >> q) & 1u) key[q] = dense_key(p, n, j4 + q);
+        }
+      }
+      const u32 top = max(max(key[0], key[1]), max(key[2], key[3]));
+      if (PER_THREAD) {  // f by the threads concerned only (no warp-wide primitive in it)
+        if (top >= min_key) f(j4, key, in);
+      } else if (__any_sync(kFull, top >= min_key)) {
+        f(j4, key, in);
+      }
+    }
+    if (PER_THREAD) {  // the hook by all lanes, converged, once per step
+      __syncwarp();
+      after();
+    }
+  }
+}
+
+__device__ __forceinline__ int dense_seg_of_index(const int64_t* seg_end, int n_seg, int64_t j) {
+  int lo = 0, hi = n_seg - 1;  // the first segment whose end lies beyond j
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (seg_end[mid] <= j) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ SegState load_seg(const DenseArgs& a, int n, int s) {  // written by other blocks of this launch
+  const uint4* q = reinterpret_cast<const uint4*>(a.seg + (size_t)n * a.n_seg + s);
+  const uint4 v = __ldcg(q), x = __ldcg(q + 1);
+  SegState r;
+  r.prefix = v.x; r.need = v.y; r.ties = v.z; r.mode = v.w;
+  r.lo = x.x; r.boff = x.y; r.bfill = x.z; r.pad = x.w;
+  return r;
+}
+
+// The tile `w` of the run of tiles the flagged workers have together: worker, segment and index range.
+struct DenseTile {
+  int n, s;
+  int64_t t;       // tile number inside the worker's row
+  int64_t t0, t1;  // coordinates
+};
+
+__device__ __forceinline__ DenseTile dense_tile(const DenseArgs& a, const u32* s_flagged, int64_t w) {
+  DenseTile r;
+  const int64_t f = w / a.tiles;
+  r.n = (int)s_flagged[f];
+  r.t = w - f * a.tiles;
+  r.s = dense_seg_of_tile(a.seg_tile0, a.n_seg, r.t);
+  const int64_t begin = r.s ? a.seg_end[r.s - 1] : 0;
+  r.t0 = begin + (r.t - a.seg_tile0[r.s]) * kDenseTile;
+  r.t1 = r.t0 + kDenseTile < a.seg_end[r.s] ? r.t0 + kDenseTile : a.seg_end[r.s];
+  return r;
+}
+
+// Drop from a warp's list the entries whose index is set in `marks` (the previous support): the probes are issued
+// four per lane at a time, so the warp waits for memory a few times per call, not once per entry.  Returns the
+// number kept (compacted to the front, order preserved).
+__device__ __forceinline__ u32 warp_drop_marked(u64* list, u32 total, const u32* marks, int lane) {
+  u32 kept = 0;
+#pragma unroll 1
+  for (u32 r0 = 0; r0 < total; r0 += 128) {
+    u64 ent[4];
+    u32 word[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const u32 i = r0 + (u32)r * 32 + lane;
+      ent[r] = i < total ? list[i] : 0ull;
+      word[r] = i < total ? __ldg(&marks[composite_idx(ent[r]) >> 5]) : 0u;
+    }
+    __syncwarp();  // every lane has read its entries before any is overwritten
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const u32 i = r0 + (u32)r * 32 + lane;
+      const bool keep = i < total && !((word[r] >> (composite_idx(ent[r]) & 31)) & 1u);
+      const u32 m = __ballot_sync(kFull, keep);
+      if (keep) list[kept + __popc(m & ((1u << lane) - 1u))] = ent[r];  // kept <= r0 + 32 r: behind the reads
+      kept += __popc(m);
+    }
+    __syncwarp();
+  }
+  return kept;
+}
+
+// A warp's staging list in shared memory (kWarpList composites): entries are added in ballot order and written out
+// to a global list, whose fill counter one lane advances, before the list can overflow.
+__device__ __forceinline__ void stage_add(u64* list, u32& count, bool pred, u64 value, int lane) {
+  const u32 m = __ballot_sync(kFull, pred);
+  if (pred && RT_INB(count + __popc(m & ((1u << lane) - 1u)) < (u32)kWarpList))
+    list[count + __popc(m & ((1u << lane) - 1u))] = value;
+  count += __popc(m);
+}
+
+__device__ __forceinline__ void stage_flush(u64* list, u32& count, u32* fill, u64* dst, u64 cap, int lane) {
+  __syncwarp();
+  if (count) {
+    u32 base = 0;
+    if (lane == 0) base = atomicAdd(fill, count);
+    base = __shfl_sync(kFull, base, 0);
+    for (u32 i = lane; i < count; i += 32)
+      if (RT_INB((u64)base + i < cap)) dst[(u64)base + i] = list[i];
+  }
+  count = 0;
+  __syncwarp();
+}
+
+__global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
+  extern __shared__ __align__(16) u64 s_stage[];  // [kDenseWarps][2 * kWarpList]: per-warp staging lists
+  __shared__ __align__(16) u32 s_hist[kBins];
+  __shared__ u32 s_flagged[kDenseMaxFlagged];
+  __shared__ u32 s_scan[33];
+  __shared__ u32 s_res[3];
+  __shared__ u32 s_cnt, s_nf;
+  __shared__ u32 s_wcnt[1][kDenseWarps];
+  cg::grid_group grid = cg::this_grid();
+  const PostArgs& p = a.p;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const u32 k = (u32)p.k;
+  u64* listA = s_stage + (size_t)warp * 2 * kWarpList;  // this warp's staging space: 2 * kWarpList entries
+
+  for (int g0 = 0; g0 < a.N; g0 += kDenseMaxFlagged) {  // groups of workers; the flags are the same in every block
+    {  // the flagged workers of this group, in order
+      constexpr int kPer = kDenseMaxFlagged / kDenseThreads;  // consecutive workers per thread
+      u32 fl = 0, cnt = 0;
+#pragma unroll
+      for (int i = 0; i < kPer; ++i) {
+        const int n = g0 + kPer * tid + i;
+        if (n < a.N && p.ctl[n].go_dense) { fl |= 1u << i; ++cnt; }
+      }
+      u32 total;
+      u32 at = block_excl_scan(cnt, s_scan, &total);
+#pragma unroll
+      for (int i = 0; i < kPer; ++i)
+        if ((fl >> i) & 1u) s_flagged[at++] = (u32)(g0 + kPer * tid + i);
+      if (tid == 0) s_nf = total;
+      __syncthreads();
+    }
+    const int64_t nf = s_nf;
+    if (nf == 0) continue;  // the same decision in every block: no barrier is skipped by some and taken by others
+    const int64_t total_tiles = nf * a.tiles;
+    const int64_t per = (total_tiles + gridDim.x - 1) / gridDim.x;
+    const int64_t w_begin = (int64_t)blockIdx.x * per < total_tiles ? (int64_t)blockIdx.x * per : total_tiles;
+    const int64_t w_end = w_begin + per < total_tiles ? w_begin + per : total_tiles;
+    const int64_t nsegs = nf * a.n_seg;
+
+    // One histogram pass over this block's tiles.  which(seg state) says whether a segment takes part; the entries
+    // counted are those with key >= lo (first digit) or whose higher digits equal the prefix (later digits).
+    auto hist_pass = [&](int lv, u32 want_mode) {
+      const int shf = lv == 0 ? 19 : (lv == 1 ? 7 : 0);  // digits of 12, 12 and 7 bits
+      const int width = lv == 2 ? 7 : 12;
+      const u32 nbm = (1u << width) - 1u;
+      int cur_n = -1, cur_s = -1;
+      bool dirty = false;
+      SegState st;
+      st.mode = ~0u;
+      for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
+      __syncthreads();
+      for (int64_t w = w_begin; w < w_end; ++w) {
+        const DenseTile t = dense_tile(a, s_flagged, w);
+        if (t.n != cur_n || t.s != cur_s) {
+          if (dirty) {
+            __syncthreads();
+            flush_hist(s_hist, a.dhist + ((size_t)cur_n * a.n_seg + cur_s) * kBins, kBins);
+            __syncthreads();
+            for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
+            __syncthreads();
+            dirty = false;
+          }
+          cur_n = t.n; cur_s = t.s;
+          st = load_seg(a, t.n, t.s);  // nothing writes it during this pass
+        }
+        if (st.mode != want_mode) continue;  // the same in every thread of the block
+        dirty = true;
+        const u32 floor_key = lv == 0 ? st.lo : st.prefix << (shf + width);  // no entry below it is counted
+        auto count = [&](int64_t j4, const u32 (&key)[4], const bool (&in)[4]) {
+          bool use[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            use[q] = in[q] && (lv == 0 ? key[q] >= st.lo : (key[q] >> (shf + width)) == st.prefix);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) hist_add_aggregated(s_hist, use[q], (key[q] >> shf) & nbm);
+        };
+        if (lv == 0 && st.lo != 0u) {
+          // with a lower bound few entries count: the threads that hold one add it themselves
+          dense_walk<true, true>(p, t.n, t.t0, t.t1, floor_key, [&](int64_t j4, const u32 (&key)[4], const bool (&in)[4]) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              if (in[q] && key[q] >= st.lo) atomicAdd(&s_hist[key[q] >> 19], 1u);
+          });
+        } else if (lv == 0) {
+          dense_walk<true>(p, t.n, t.t0, t.t1, floor_key, count);  // (the previous support is counted from the override list)
+        } else {
+          dense_walk<false>(p, t.n, t.t0, t.t1, floor_key, count);
+        }
+      }
+      __syncthreads();
+      if (dirty) flush_hist(s_hist, a.dhist + ((size_t)cur_n * a.n_seg + cur_s) * kBins, kBins);
+      if (lv == 0 && p.use_marks) {
+        // the entries of the previous support, which the walk above left out: their scores come from the override
+        // list (index order), one lane per entry, straight into the segments' histograms in global memory
+        for (int64_t f = 0; f < nf; ++f) {
+          const int n = (int)s_flagged[f];
+          const int32_t* pi = p.prev_idx + (size_t)n * p.k;
+          const u32* okey = p.ovr_key + (size_t)n * p.k;
+          for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + (tid & ~31); i0 < p.k; i0 += (int64_t)gridDim.x * blockDim.x) {
+            const int64_t i = i0 + lane;
+            bool use = i < p.k;
+            const int32_t j = use ? pi[i] : 0;
+            const u32 key = use ? __ldcg(&okey[i]) : 0u;
+            const int s = a.n_seg > 1 ? dense_seg_of_index(a.seg_end, a.n_seg, j) : 0;
+            bool take_back = false;
+            u32 lo_seg = 0;
+            if (use) {
+              const SegState st = load_seg(a, n, s);
+              take_back = st.mode == want_mode;
+              lo_seg = st.lo;
+              use = take_back && key >= st.lo;
+            }
+            u32* hist = a.dhist + ((size_t)n * a.n_seg + s) * kBins;
+            u32* target = hist + (key >> 19);
+            const u32 act = __ballot_sync(kFull, use);
+            if (use) {  // lanes that count into the same bin add once
+              const u32 peers = __match_any_sync(act, (u64)(uintptr_t)target);
+              if (lane == __ffs(peers) - 1) atomicAdd(target, (u32)__popc(peers));
+            }
+            // the walk counted the entry under bits(|a|): take that back (the sums are what matters: a bin may
+            // pass through "negative" values on the way)
+            if (take_back) {
+              const u32 ka = __float_as_uint(p.eps[(size_t)n * p.ld + j]) & 0x7FFFFFFFu;
+              if (ka >= lo_seg) atomicSub(hist + (ka >> 19), 1u);
+            }
+          }
+        }
+      }
+    };
+
+    // Per segment that takes part: load its histogram (clearing it for the next use) and find the bin of the
+    // need-th largest.  done(st, b, above, in_bin) runs in thread 0 and updates the state; b == kFull: the
+    // histogram holds fewer than `need` entries.
+    auto find_pass = [&](int lv, u32 want_mode, auto done) {
+      for (int64_t v = blockIdx.x; v < nsegs; v += gridDim.x) {
+        const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
+        const SegState old = load_seg(a, n, s);
+        if (old.mode != want_mode) continue;  // the same in every thread of the block
+        u32* gh = a.dhist + ((size_t)n * a.n_seg + s) * kBins;
+        __syncthreads();
+        for (int i = tid; i < kBins; i += blockDim.x) {
+          s_hist[i] = __ldcg(&gh[i]);
+          gh[i] = 0;  // ready for the next digit, and for the next launch
+        }
+        const u32 need = lv ? old.need : (u32)(a.seg_kpre[s + 1] - a.seg_kpre[s]);
+        __syncthreads();
+        block_find_from_top(s_hist, kBins, need, s_scan, s_res);
+        if (tid == 0) done(n, s, old, need, s_res[0], s_res[1], s_res[0] == kFull ? 0u : s_hist[s_res[0]]);
+        __syncthreads();
+      }
+    };
+
+    // ---- set-up: the lower bound each segment starts with ----
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + tid; v < nsegs; v += (int64_t)gridDim.x * blockDim.x) {
+      const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
+      u32 lo;
+      if (a.layered) {
+        const u32 thr = a.seg_thr[(size_t)n * a.n_seg + s];  // lower edge of the bin of last round's threshold
+        lo = thr > kHintMargin ? thr - kHintMargin : 0u;
+      } else {
+        // the sampled cutoff as it is when the path was asked for; an octave lower when that cutoff has just left
+        // too few entries above it
+        const u32 hint = p.ctl[n].hint;
+        lo = hint == kFull ? 0u : (p.ctl[n].force_dense ? hint : (hint > kOctave ? hint - kOctave : 0u));
+      }
+      SegState st;
+      st.prefix = 0; st.need = 0; st.ties = 0; st.mode = kSegRetry; st.lo = lo; st.boff = 0; st.bfill = 0; st.pad = 0;
+      a.seg[(size_t)n * a.n_seg + s] = st;
+    }
+    grid.sync();
+
+    // ---- (A) first digit; once more with lo = 0 for the segments whose hint was too high ----
+    for (int attempt = 0; attempt < 2; ++attempt) {
+      hist_pass(0, kSegRetry);
+      grid.sync();
+      find_pass(0, kSegRetry, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin) {
+        SegState* st = a.seg + (size_t)n * a.n_seg + s;
+        if (b == kFull) {
+          if (old.lo == 0u) {  // fewer than k entries in the whole segment: cannot happen
+            atomicOr(&p.gctl->dense_flags, kFlagBad);
+            st->mode = kSegList; st->prefix = 0; st->need = 0; st->ties = 0;
+          } else {
+            st->lo = 0u;  // stays kSegRetry
+            atomicOr(&p.gctl->dense_flags, kFlagRetry);
+          }
+          return;
+        }
+        st->prefix = b;
+        st->need = need - above;
+        st->ties = in_bin;
+        a.seg_thr[(size_t)n * a.n_seg + s] = b << 19;  // lower edge of the bin: next round's hint
+        // room for the bin's entries in the worker's B list?
+        const u32 off = atomicAdd(&p.ctl[n].bcount, in_bin);
+        if ((u64)off + in_bin <= (u64)p.stride) {
+          st->mode = kSegList;
+          st->boff = off;
+        } else {
+          st->mode = kSegRows;
+          atomicOr(&p.gctl->dense_flags, kFlagRows);
+        }
+      });
+      grid.sync();
+      if (!(__ldcg(&p.gctl->dense_flags) & kFlagRetry)) break;  // the same in every block
+      grid.sync();  // everyone has seen the flag
+      if (blockIdx.x == 0 && tid == 0) atomicAnd(&p.gctl->dense_flags, ~kFlagRetry);
+    }
+
+    // ---- (B) second pass over the rows: winners above the bin, and the bin's own entries to their list ----
+    {
+      int cur_n = -1, cur_s = -1;
+      // During the walk a thread that holds an entry at or above the bin's lower edge puts it into its warp's
+      // staging list itself (one shared-memory counter).  When the list is half full, or the segment changes, the
+      // warp writes it out: entries on the previous support are dropped (their scores come from the override list),
+      // entries above the bin win (mask bit, winner list), the bin's own go to the segment's in-bin list.
+      u64* list = listA;  // both halves of the warp's staging space: 2 * kWarpList entries
+      constexpr u32 kCap = 2u * kWarpList;
+      auto marked = [&](int n, u32 j) {
+        return p.use_marks && ((__ldg(p.mask_old + (size_t)n * p.W + (j >> 5)) >> (j & 31)) & 1u);
+      };
+      auto place = [&](int n, int s, const SegState& sg, u64 c, bool live) {  // all lanes of the warp; live: this lane has an entry
+        const bool isA = live && (u32)(c >> 51) > sg.prefix;  // key >> 19
+        const bool isB = live && !isA;
+        const u32 mA = __ballot_sync(kFull, isA), mB = __ballot_sync(kFull, isB);
+        u32 baseA = 0, baseB = 0;
+        if (lane == 0 && mA) baseA = atomicAdd(&p.ctl[n].acount, (u32)__popc(mA));
+        if (lane == 0 && mB) baseB = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, (u32)__popc(mB));
+        baseA = __shfl_sync(kFull, baseA, 0);
+        baseB = __shfl_sync(kFull, baseB, 0);
+        const u32 lt = (1u << lane) - 1u;
+        if (isA) {
+          set_winner(p.mask_new + (size_t)n * p.W, composite_idx(c), p.d);
+          const u32 pos = baseA + __popc(mA & lt);
+          if (RT_INB(pos < k)) p.candA[(size_t)n * p.stride + pos] = c;
+        }
+        if (isB) {
+          const u32 pos = baseB + __popc(mB & lt);
+          if (RT_INB(pos < sg.ties)) p.candB[(size_t)n * p.stride + sg.boff + pos] = c;
+        }
+      };
+      auto flush = [&](int n, int s, const SegState& sg) {  // every lane of the warp
+        __syncwarp();
+        u32 c = *reinterpret_cast<volatile u32*>(&s_wcnt[0][warp]);
+        c = c < kCap ? c : kCap;
+        if (p.use_marks && c) c = warp_drop_marked(list, c, p.mask_old + (size_t)n * p.W, lane);
+        for (u32 i0 = 0; i0 < c; i0 += 32) place(n, s, sg, i0 + lane < c ? list[i0 + lane] : 0ull, i0 + lane < c);
+        __syncwarp();
+        if (lane == 0) s_wcnt[0][warp] = 0;
+        __syncwarp();
+      };
+      // A region dense with winners can fill the list within one step of the walk; an entry that finds it full
+      // goes out by itself.
+      auto direct = [&](int n, int s, const SegState& sg, u64 c) {
+        const u32 j = composite_idx(c);
+        if (marked(n, j)) return;
+        if ((u32)(c >> 51) > sg.prefix) {
+          set_winner(p.mask_new + (size_t)n * p.W, j, p.d);
+          const u32 pos = atomicAdd(&p.ctl[n].acount, 1u);
+          if (RT_INB(pos < k)) p.candA[(size_t)n * p.stride + pos] = c;
+        } else {
+          const u32 pos = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, 1u);
+          if (RT_INB(pos < sg.ties)) p.candB[(size_t)n * p.stride + sg.boff + pos] = c;
+        }
+      };
+      if (lane == 0) s_wcnt[0][warp] = 0;
+      __syncwarp();
+      SegState st;
+      st.mode = ~0u;
+      for (int64_t w = w_begin; w < w_end; ++w) {
+        const DenseTile t = dense_tile(a, s_flagged, w);
+        if (t.n != cur_n || t.s != cur_s) {
+          if (cur_n >= 0 && st.mode == kSegList) flush(cur_n, cur_s, st);
+          cur_n = t.n; cur_s = t.s;
+          st = load_seg(a, t.n, t.s);  // but for its fill counter, nothing writes it during this pass
+        }
+        if (st.mode != kSegList) continue;  // the same in every thread of the block
+        const u32 floor_key = max(st.prefix << 19, st.lo);  // nothing below it is a winner or in the bin
+        dense_walk<true, true>(p, t.n, t.t0, t.t1, floor_key,
+          [&](int64_t j4, const u32 (&key)[4], const bool (&in)[4]) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              if (!in[q] || key[q] < floor_key) continue;
+              const u64 c = make_composite(key[q], (u32)(j4 + q));
+              const u32 at = atomicAdd(&s_wcnt[0][warp], 1u);
+              if (at < kCap) list[at] = c;
+              else direct(t.n, t.s, st, c);
+            }
+          },
+          [&]() {
+            if (*reinterpret_cast<volatile u32*>(&s_wcnt[0][warp]) >= kCap / 2u) flush(t.n, t.s, st);
+          });
+      }
+      if (cur_n >= 0 && st.mode == kSegList) flush(cur_n, cur_s, st);
+      u32 cntA = 0;  // from here on the lists are filled by ballot: warp-uniform fill
+      auto flush_A2 = [&](int n) {
+        stage_flush(listA, cntA, &p.ctl[n].acount, p.candA + (size_t)n * p.stride, (u64)k, lane);
+      };
+      if (p.use_marks) {  // the same for the entries of the previous support, from the override list
+        for (int64_t f = 0; f < nf; ++f) {
+          const int n = (int)s_flagged[f];
+          const int32_t* pi = p.prev_idx + (size_t)n * p.k;
+          const u32* okey = p.ovr_key + (size_t)n * p.k;
+          u32* mask = p.mask_new + (size_t)n * p.W;
+          for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + (tid & ~31); i0 < p.k; i0 += (int64_t)gridDim.x * blockDim.x) {
+            const int64_t i = i0 + lane;
+            const bool live = i < p.k;
+            const int32_t j = live ? pi[i] : 0;
+            const u32 key = live ? __ldcg(&okey[i]) : 0u;
+            const int s = a.n_seg > 1 ? dense_seg_of_index(a.seg_end, a.n_seg, j) : 0;
+            bool win = false, bin = false;
+            SegState st;
+            st.boff = 0; st.ties = 0;
+            if (live) {
+              st = load_seg(a, n, s);
+              if (st.mode == kSegList) {
+                win = (key >> 19) > st.prefix;
+                bin = (key >> 19) == st.prefix && key >= st.lo;
+              }
+            }
+            const u64 c = make_composite(key, (u32)j);
+            if (win) set_winner(mask, (u32)j, p.d);
+            if (bin) {
+              const u32 pos = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, 1u);
+              if (RT_INB(pos < st.ties)) p.candB[(size_t)n * p.stride + st.boff + pos] = c;
+            }
+            if (__any_sync(kFull, win)) {
+              stage_add(listA, cntA, win, c, lane);
+              if (cntA >= (u32)(kWarpList - 32)) flush_A2(n);
+            }
+          }
+          flush_A2(n);
+        }
+      }
+    }
+    const u32 flags0 = __ldcg(&p.gctl->dense_flags);  // written before the last barrier
+    if (flags0 & kFlagRows) hist_pass(1, kSegRows);
+    grid.sync();
+
+    // ---- (C) per list segment: the `need` largest composites of its in-bin list win ----
+    for (int64_t v = blockIdx.x; v < nsegs; v += gridDim.x) {
+      const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
+      const SegState st = load_seg(a, n, s);
+      if (st.mode != kSegList || st.need == 0u) continue;  // the same in every thread of the block
+      const u64* list = p.candB + (size_t)n * p.stride + st.boff;
+      u32* mask = p.mask_new + (size_t)n * p.W;
+      const u32 count = st.ties;
+      if (st.bfill != count) {
+        if (tid == 0) atomicOr(&p.gctl->dense_flags, kFlagBad);
+        continue;
+      }
+      // the need-th largest composite, byte by byte (the list stays where it is)
+      u32 need = st.need;
+      u64 prefix = 0ull;
+      bool bad = false;
+      if (need < count) {
+        for (int shift = 56; shift >= 0 && !bad; shift -= 8) {
+          __syncthreads();
+          for (int i = tid; i < 256; i += blockDim.x) s_hist[i] = 0;
+          __syncthreads();
+          for (u32 i = tid; i < count; i += blockDim.x) {
+            const u64 c = __ldcg(&list[i]);
+            if (shift == 56 || (c >> (shift + 8)) == prefix) atomicAdd(&s_hist[(u32)(c >> shift) & 255u], 1u);
+          }
+          __syncthreads();
+          block_find_from_top(s_hist, 256, need, s_scan, s_res);
+          const u32 b = s_res[0], above = s_res[1];
+          if (b == kFull) { bad = true; break; }  // the same in every thread
+          need -= above;
+          prefix = (prefix << 8) | (u64)b;
+        }
+      }
+      if (bad) {
+        if (tid == 0) atomicOr(&p.gctl->dense_flags, kFlagBad);
+        continue;
+      }
+      // winners: at or above that composite (every entry if all are needed); they join the worker's winner list
+      __syncthreads();
+      if (tid == 0) s_cnt = atomicAdd(&p.ctl[n].acount, st.need);
+      __syncthreads();
+      const u32 abase = s_cnt;
+      u64* A = p.candA + (size_t)n * p.stride;
+      u32 carry = 0;
+      for (u32 i0 = 0; i0 < count; i0 += blockDim.x) {
+        const u32 i = i0 + tid;
+        const u64 c = i < count ? __ldcg(&list[i]) : 0ull;
+        const bool won = i < count && c >= prefix;
+        u32 total;
+        const u32 at = block_excl_scan(won ? 1u : 0u, s_scan, &total);
+        if (won) {
+          set_winner(mask, composite_idx(c), p.d);
+          if (RT_INB((u64)abase + carry + at < (u64)k)) A[(u64)abase + carry + at] = c;
+        }
+        carry += total;
+      }
+    }
+    if (flags0 & kFlagRows) {
+      find_pass(1, kSegRows, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin) {
+        SegState* st = a.seg + (size_t)n * a.n_seg + s;
+        if (b == kFull) { atomicOr(&p.gctl->dense_flags, kFlagBad); b = 0; above = 0; }
+        st->prefix = (old.prefix << 12) | b;
+        st->need = need - above;
+        st->ties = in_bin;
+      });
+      grid.sync();
+      hist_pass(2, kSegRows);
+      grid.sync();
+      find_pass(2, kSegRows, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin) {
+        SegState* st = a.seg + (size_t)n * a.n_seg + s;
+        if (b == kFull) { atomicOr(&p.gctl->dense_flags, kFlagBad); b = 0; above = 0; }
+        st->prefix = (old.prefix << 7) | b;
+        st->need = need - above;
+        st->ties = in_bin;
+        if (in_bin > need - above) atomicOr(&p.gctl->dense_flags, kFlagOrdered);
+      });
+      grid.sync();
+      const u32 flags1 = __ldcg(&p.gctl->dense_flags);
+
+      // ties in index order: per tile the number of entries equal to the threshold key T, then, per segment, the
+      // number of them in lower tiles
+      if (flags1 & kFlagOrdered) {
+        for (int64_t w = w_begin; w < w_end; ++w) {
+          const DenseTile t = dense_tile(a, s_flagged, w);
+          const SegState st = load_seg(a, t.n, t.s);
+          if (st.mode != kSegRows || st.ties <= st.need) continue;  // the same in every thread of the block
+          if (tid == 0) s_cnt = 0;
+          __syncthreads();
+          u32 mine = 0;
+          dense_walk<false>(p, t.n, t.t0, t.t1, st.prefix, [&](int64_t, const u32 (&key)[4], const bool (&in)[4]) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) mine += (in[q] && key[q] == st.prefix) ? 1u : 0u;
+          });
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(kFull, mine, o);
+          if (lane == 0 && mine) atomicAdd(&s_cnt, mine);
+          __syncthreads();
+          if (tid == 0) a.tile_ties[2 * ((size_t)t.n * a.tiles + t.t)] = s_cnt;
+          __syncthreads();
+        }
+        grid.sync();
+        for (int64_t v = blockIdx.x; v < nsegs; v += gridDim.x) {
+          const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
+          const SegState st = load_seg(a, n, s);
+          if (st.mode != kSegRows || st.ties <= st.need) continue;  // the same in every thread of the block
+          u32* tt = a.tile_ties + 2 * (size_t)n * a.tiles;
+          u32 carry = 0;
+          for (int64_t c0 = a.seg_tile0[s]; c0 < a.seg_tile0[s + 1]; c0 += blockDim.x) {
+            const int64_t c = c0 + tid;
+            const u32 mine = c < a.seg_tile0[s + 1] ? __ldcg(&tt[2 * c]) : 0u;
+            u32 total;
+            const u32 before = block_excl_scan(mine, s_scan, &total);
+            if (c < a.seg_tile0[s + 1]) tt[2 * c + 1] = carry + before;
+            carry += total;
+          }
+        }
+        grid.sync();
+      }
+      // last pass over the rows of those segments: winners are the entries above T and the ties that are taken
+      {
+        u32 cntA = 0;
+        int cur_n = -1;
+        auto flush_A = [&](int n) {
+          stage_flush(listA, cntA, &p.ctl[n].acount, p.candA + (size_t)n * p.stride, (u64)k, lane);
+        };
+        for (int64_t w = w_begin; w < w_end; ++w) {
+          const DenseTile t = dense_tile(a, s_flagged, w);
+          if (t.n != cur_n) {
+            if (cur_n >= 0) flush_A(cur_n);
+            cur_n = t.n;
+          }
+          const SegState st = load_seg(a, t.n, t.s);
+          if (st.mode != kSegRows) continue;  // the same in every thread of the block
+          const u32 T = st.prefix, need = st.need;
+          // all of the tile's ties win, none of them, or (one tile per segment at most) the first few in index order
+          bool all_win = st.ties <= need, none_win = false;
+          u32 tie_rank = 0;
+          if (!all_win) {
+            const u32 here = __ldcg(&a.tile_ties[2 * ((size_t)t.n * a.tiles + t.t)]);
+            tie_rank = __ldcg(&a.tile_ties[2 * ((size_t)t.n * a.tiles + t.t) + 1]);
+            all_win = tie_rank + here <= need;
+            none_win = tie_rank >= need;
+          }
+          const bool in_order = !all_win && !none_win;
+          u32* mask = p.mask_new + (size_t)t.n * p.W;
+          dense_walk<false>(p, t.n, t.t0, t.t1, in_order ? 0u : T, [&](int64_t j4, const u32 (&key)[4], const bool (&in)[4]) {
+            bool win[4];
+            u32 eq = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              win[q] = in[q] && (key[q] > T || (key[q] == T && all_win));
+              eq += (in[q] && key[q] == T) ? 1u : 0u;
+            }
+            if (in_order) {  // the same in every thread of the block; threads hold consecutive quads
+              u32 total;
+              u32 r = tie_rank + block_excl_scan(eq, s_scan, &total);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                if (in[q] && key[q] == T) {
+                  win[q] = r < need;
+                  ++r;
+                }
+              }
+              tie_rank += total;
+            }
+            u32 bits = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) bits |= win[q] ? (1u << q) : 0u;
+            if (bits && RT_INB(j4 + 3 < p.W * 32)) atomicOr(&mask[j4 >> 5], bits << (j4 & 31));
+            if (__any_sync(kFull, bits != 0u)) {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) stage_add(listA, cntA, win[q], make_composite(key[q], (u32)(j4 + q)), lane);
+              if (cntA >= (u32)(kWarpList - 128)) flush_A(t.n);
+            }
+          });
+        }
+        if (cur_n >= 0) flush_A(cur_n);
+      }
+    }
+    grid.sync();
+    // every flagged worker must have gathered exactly k winners
+    const u32 flags2 = __ldcg(&p.gctl->dense_flags);
+    for (int64_t f = blockIdx.x; f < nf; f += gridDim.x) {
+      if (tid == 0) {
+        const int n = (int)s_flagged[f];
+        if ((flags2 & kFlagBad) || __ldcg(&p.ctl[n].acount) != k) atomicOr(&p.gctl->err, kErrDenseSelect);
+        p.ctl[n].took_dense = 1u;
+      }
+    }
+
+    if (a.finish) {
+      // ---- ranks and emission, as in k_post: per-quad prefix counts of the mask, segment bases, then every
+      //      winner looks its rank up and writes its pair ----
+      const int nw = blockDim.x >> 5;
+      const int64_t U = p.W >> 3;
+      const int64_t seg_units = (U + a.emit_segments - 1) / a.emit_segments;
+      for (int64_t it = (int64_t)blockIdx.x * nw + warp; it < nf * a.emit_segments; it += (int64_t)gridDim.x * nw)
+        post_prefix_segment(p, (int)s_flagged[it / a.emit_segments], (u32)(it % a.emit_segments), seg_units, lane);
+      grid.sync();
+      u32* s_segbase = s_hist;
+      for (int64_t f = 0; f < nf; ++f) {
+        const int n = (int)s_flagged[f];
+        constexpr int kSegPer = kMaxSegments / kDenseThreads;  // consecutive mask segments per thread
+        u32 mine[kSegPer], sum = 0, total;
+#pragma unroll
+        for (int i = 0; i < kSegPer; ++i) {
+          const u32 sg = (u32)(kSegPer * tid + i);
+          mine[i] = sg < a.emit_segments ? __ldcg(&p.segtot[(size_t)n * kMaxSegments + sg]) : 0u;
+          sum += mine[i];
+        }
+        u32 base = block_excl_scan(sum, s_scan, &total);
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kSegPer; ++i) {
+          const u32 sg = (u32)(kSegPer * tid + i);
+          if (sg < a.emit_segments) {
+            s_segbase[sg] = base;
+            if (blockIdx.x == 0) p.segbase[(size_t)n * kMaxSegments + sg] = base;  // for k_aggregate
+          }
+          base += mine[i];
+        }
+        __syncthreads();
+        if (total != k) {
+          if (blockIdx.x == 0 && tid == 0) atomicOr(&p.gctl->err, kErrCountMismatch);
+        } else {
+          post_emit(p, n, blockIdx.x * blockDim.x + tid, gridDim.x * blockDim.x, 0u, 0u, true, 0u, 0u, 0u, s_segbase,
+                    seg_units);
+        }
+        __syncthreads();
+      }
+    }
+    grid.sync();  // everyone has read the flag word before it is cleared for the next group and the next launch
+    if (blockIdx.x == 0 && tid == 0) p.gctl->dense_flags = 0u;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // k_aggregate: g = sum_n omega_n * ghat_n with the workers added in the order n = 0..N-1.
 // One thread per pair sent this round: the pair of the highest-numbered worker that sent index j
 // owns g[j]; it looks the lower workers' values up (mask quad, prefix counts, value) and adds them
@@ -1708,6 +2516,8 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   int64_t ld, W, capA, stride;
+  int64_t n_seg, tiles;  // segments of a row (layers; 1 in the plain mode) and k_dense tiles per row
+  size_t off_dhist, off_seg_thr, off_seg, off_tile_ties, off_seg_end, off_seg_kpre, off_seg_tile0;
   size_t off_eps, off_g, off_mask[2], off_ctl, off_gctl, off_shist, zero_end, off_skeys, off_qprefix, off_segtot, off_segbase, off_ghist, off_btot, off_idx[2], off_val[2],
       off_ovr_key, off_ovr_comp, off_candA, off_candB, off_omega, off_stage_g, off_stage_idx,
       off_stage_val, total;
@@ -1722,7 +2532,37 @@ bool valid_problem(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
   if (pr->omega)
     for (int n = 0; n < N; ++n)
       if (!isfinite(pr->omega[n])) return false;
+  if (pr->n_layers < 0 || pr->n_layers > 65536) return false;
+  if (pr->n_layers > 0) {  // contiguous layers that cover [0, d); the per-layer k add up to k
+    if (!pr->layer_end || !pr->layer_k) return false;
+    int64_t begin = 0, ksum = 0;
+    for (int l = 0; l < pr->n_layers; ++l) {
+      if (pr->layer_end[l] <= begin || pr->layer_end[l] > d) return false;
+      if (pr->layer_k[l] < 1 || pr->layer_k[l] > pr->layer_end[l] - begin) return false;
+      ksum += pr->layer_k[l];
+      begin = pr->layer_end[l];
+    }
+    if (begin != d || ksum != k) return false;
+  }
   return true;
+}
+
+// Segment tables of k_dense on the host: ends, exclusive prefix sums of the per-segment k, first tile of each
+// segment (tiles of kDenseTile coordinates never straddle a segment).  Arrays of n_seg, n_seg + 1, n_seg + 1.
+int64_t segment_tables(int64_t d, int64_t k, const regtopk_params* pr, int64_t* seg_end, int64_t* seg_kpre,
+                       int64_t* seg_tile0) {
+  const int64_t n_seg = pr->n_layers > 0 ? pr->n_layers : 1;
+  int64_t begin = 0, kpre = 0, tile = 0;
+  for (int64_t s = 0; s < n_seg; ++s) {
+    const int64_t end = pr->n_layers > 0 ? pr->layer_end[s] : d;
+    const int64_t ks = pr->n_layers > 0 ? pr->layer_k[s] : k;
+    if (seg_end) { seg_end[s] = end; seg_kpre[s] = kpre; seg_tile0[s] = tile; }
+    kpre += ks;
+    tile += (end - begin + kDenseTile - 1) / kDenseTile;
+    begin = end;
+  }
+  if (seg_end) { seg_kpre[n_seg] = kpre; seg_tile0[n_seg] = tile; }
+  return tile;
 }
 
 Layout make_layout(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
@@ -1746,7 +2586,16 @@ Layout make_layout(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
   L.off_ctl = take((size_t)N * sizeof(WorkerCtl));
   L.off_gctl = take(sizeof(GlobalCtl));
   L.off_shist = take((size_t)N * kSampleBins * 4);
+  L.n_seg = pr->n_layers > 0 ? pr->n_layers : 1;
+  L.tiles = segment_tables(d, k, pr, nullptr, nullptr, nullptr);
+  L.off_dhist = take((size_t)N * L.n_seg * kBins * 4);
+  L.off_seg_thr = take((size_t)N * L.n_seg * 4);
   L.zero_end = o;
+  L.off_seg = take((size_t)N * L.n_seg * sizeof(SegState));
+  L.off_tile_ties = take((size_t)N * L.tiles * 8);
+  L.off_seg_end = take((size_t)L.n_seg * 8);
+  L.off_seg_kpre = take((size_t)(L.n_seg + 1) * 8);
+  L.off_seg_tile0 = take((size_t)(L.n_seg + 1) * 8);
   L.off_skeys = take((size_t)N * kSampleMax * 4);
   L.off_qprefix = take((size_t)N * (L.W / 4) * 4);
   L.off_segtot = take((size_t)N * kMaxSegments * 4);
@@ -1777,6 +2626,7 @@ constexpr int kMaxProfile = 4096;
 #define REGTOPK_MANY_PAIRS 262144
 #endif
 constexpr int64_t kManyPairs = REGTOPK_MANY_PAIRS;  // N*k from which the list phases run in wide mode
+constexpr int64_t kGridDenseCoords = 1ll << 28;     // N*d from which the dense exact path runs on the whole grid
 
 }  // namespace
 
@@ -1795,6 +2645,10 @@ struct regtopk_ctx {
   int num_sms;
   int cluster;       // blocks per worker in k_post
   int many_pairs;    // N*k is large (or the testing flag is set): wide kernels and pair-mode emission
+  int layered;       // one selection per layer: every worker takes the dense path of k_dense every round
+  int grid_dense;    // workers that need the dense exact path are served by k_dense, not by their k_post cluster
+  int dense_blocks;  // co-resident blocks of k_dense (its grid)
+  uint64_t layer_hash;
   int stream_blocks[5];
   int64_t launches;
   int profiling;
@@ -1820,6 +2674,7 @@ int after_launch(regtopk_ctx* c) {
 }
 
 size_t sample_smem() { return (size_t)kSamplePadded * sizeof(u32); }
+size_t dense_smem() { return (size_t)2 * kDenseWarps * kWarpList * sizeof(u64); }
 
 // Launch configuration: `blocks` blocks of `threads`, optionally in clusters, always with programmatic
 // stream serialization (see grid_dependency_begin).  attr must have room for two attributes.
@@ -1971,6 +2826,23 @@ int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const reg
   c->num_sms = sms > 0 ? sms : 148;
   c->cluster = choose_cluster(N);
   c->many_pairs = (k * (int64_t)N >= kManyPairs || (params->flags & REGTOPK_FLAG_FORCE_WIDE_LISTS)) ? 1 : 0;
+  c->layered = params->n_layers > 0 ? 1 : 0;
+  // Rows large enough for one more (empty) kernel per round to go unnoticed get the full-grid dense path; on small
+  // problems a worker's own cluster scans its row, which costs the common round nothing.
+  c->grid_dense = (c->layered || c->many_pairs || (params->flags & REGTOPK_FLAG_GRID_DENSE_SELECT) ||
+                   d * (int64_t)N >= kGridDenseCoords) ? 1 : 0;
+  {
+    int per_sm = 0;
+    if (cudaFuncSetAttribute(k_dense, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dense_smem()) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_dense, kDenseThreads, dense_smem()) != cudaSuccess ||
+        per_sm < 1) {
+      cudaGetLastError();
+      per_sm = 1;
+    }
+    int64_t blocks = (int64_t)per_sm * c->num_sms;
+    if (blocks > (int64_t)N * L.tiles) blocks = (int64_t)N * L.tiles;
+    c->dense_blocks = (int)(blocks < 1 ? 1 : blocks);
+  }
   float* om = static_cast<float*>(malloc(sizeof(float) * N));
   if (!om) { free(c); return REGTOPK_ERR_INVALID_ARG; }
   for (int n = 0; n < N; ++n) om[n] = params->omega ? params->omega[n] : 1.0f / (float)N;
@@ -1979,8 +2851,27 @@ int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const reg
   if (rc == REGTOPK_OK)
     rc = note_cuda(c, cudaMemcpyAsync(c->ws + L.off_omega, om, sizeof(float) * N,
                                       cudaMemcpyHostToDevice, c->stream));
+  int64_t* seg = static_cast<int64_t*>(malloc(sizeof(int64_t) * (3 * (size_t)L.n_seg + 2)));
+  if (!seg) { free(om); free(c); return REGTOPK_ERR_INVALID_ARG; }
+  {
+    int64_t* seg_end = seg;
+    int64_t* seg_kpre = seg + L.n_seg;
+    int64_t* seg_tile0 = seg + 2 * L.n_seg + 1;
+    segment_tables(d, k, params, seg_end, seg_kpre, seg_tile0);
+    uint64_t h = 1469598103934665603ull;  // FNV-1a over the layer table: a checkpoint must come from the same layers
+    for (int64_t i = 0; i < L.n_seg; ++i)
+      for (int64_t v : {seg_end[i], seg_kpre[i + 1]}) { h ^= (uint64_t)v; h *= 1099511628211ull; }
+    c->layer_hash = params->n_layers > 0 ? h : 0;
+    if (rc == REGTOPK_OK)
+      rc = note_cuda(c, cudaMemcpyAsync(c->ws + L.off_seg_end, seg_end, 8 * (size_t)L.n_seg, cudaMemcpyHostToDevice, c->stream));
+    if (rc == REGTOPK_OK)
+      rc = note_cuda(c, cudaMemcpyAsync(c->ws + L.off_seg_kpre, seg_kpre, 8 * ((size_t)L.n_seg + 1), cudaMemcpyHostToDevice, c->stream));
+    if (rc == REGTOPK_OK)
+      rc = note_cuda(c, cudaMemcpyAsync(c->ws + L.off_seg_tile0, seg_tile0, 8 * ((size_t)L.n_seg + 1), cudaMemcpyHostToDevice, c->stream));
+  }
   if (rc == REGTOPK_OK) rc = note_cuda(c, cudaStreamSynchronize(c->stream));
   free(om);
+  free(seg);
   if (rc != REGTOPK_OK) { free(c); return rc; }
   *out = c;
   return REGTOPK_OK;
@@ -2020,7 +2911,7 @@ int step_impl(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_i
   sa.omega = at<float>(c, L.off_omega); sa.mu = c->mu; sa.inv_y = c->inv_y; sa.ovr_key = at<u32>(c, L.off_ovr_key);
   sa.share_override = 0;
   sa.inplace = inplace ? 1 : 0;
-  sa.force_dense = (c->flags & REGTOPK_FLAG_FORCE_DENSE_SELECT) ? 1 : 0;
+  sa.force_dense = c->layered ? 1 : ((c->flags & REGTOPK_FLAG_FORCE_DENSE_SELECT) ? (c->grid_dense ? 2 : 1) : 0);
   {
     cudaLaunchConfig_t scfg;
     cudaLaunchAttribute sattr[2];
@@ -2064,6 +2955,7 @@ int step_impl(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_i
   pa.use_marks = use_marks; pa.has_stale = c->round >= 2;
   pa.pair_mode = c->many_pairs;
   pa.wide = c->many_pairs;
+  pa.grid_dense = c->grid_dense;
   // wide kernels: the grid's blocks split evenly over the workers (blockIdx.y = worker)
   cudaLaunchConfig_t wcfg;
   cudaLaunchAttribute wattr[2];
@@ -2086,6 +2978,33 @@ int step_impl(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_i
   c->launches++;
   if (le != cudaSuccess) return note_cuda(c, le);
   if ((rc = note_cuda(c, cudaGetLastError()))) return rc;
+  if (c->grid_dense) {
+    // Cooperative launch in plain stream order: it starts when k_post has completed, and returns at once unless a
+    // worker asked for the dense path.
+    DenseArgs da;
+    da.p = pa; da.N = c->N; da.n_seg = (int)L.n_seg; da.finish = pa.wide ? 0 : 1;
+    da.emit_segments = (u32)(c->cluster * (kBlockPost / 32));
+    da.tiles = L.tiles;
+    da.seg_end = at<int64_t>(c, L.off_seg_end); da.seg_kpre = at<int64_t>(c, L.off_seg_kpre);
+    da.seg_tile0 = at<int64_t>(c, L.off_seg_tile0);
+    da.dhist = at<u32>(c, L.off_dhist); da.seg = at<SegState>(c, L.off_seg); da.tile_ties = at<u32>(c, L.off_tile_ties);
+    da.seg_thr = at<u32>(c, L.off_seg_thr); da.layered = c->layered;
+    cudaLaunchConfig_t dcfg;
+    cudaLaunchAttribute dattr[1];
+    memset(&dcfg, 0, sizeof dcfg);
+    dcfg.gridDim = dim3((unsigned)c->dense_blocks, 1, 1);
+    dcfg.blockDim = dim3(kDenseThreads, 1, 1);
+    dcfg.dynamicSmemBytes = dense_smem();
+    dcfg.stream = c->stream;
+    dattr[0].id = cudaLaunchAttributeCooperative;
+    dattr[0].val.cooperative = 1;
+    dcfg.attrs = dattr;
+    dcfg.numAttrs = 1;
+    cudaError_t de = cudaLaunchKernelEx(&dcfg, k_dense, da);
+    c->launches++;
+    if (de != cudaSuccess) return note_cuda(c, de);
+    if ((rc = note_cuda(c, cudaGetLastError()))) return rc;
+  }
   if (pa.wide) {
     cudaLaunchKernelEx(&wcfg, k_wide_prefix, pa);
     if ((rc = after_launch(c))) return rc;
@@ -2184,6 +3103,7 @@ struct StateHeader {
   int64_t d, k, ld, W, round;
   int32_t N, cur, grad_dtype;
   uint32_t mu_bits, inv_y_bits;
+  uint64_t layer_hash;
 };
 constexpr uint64_t kStateMagic = 0x52544B5354415445ull;  // "RTKSTATE"
 constexpr size_t kStateHeaderBytes = 256;
@@ -2207,6 +3127,7 @@ int regtopk_state_export(regtopk_ctx* c, void* dst, size_t bytes) {
   h.N = c->N; h.cur = c->cur; h.grad_dtype = c->grad_dtype;
   memcpy(&h.mu_bits, &c->mu, 4);
   memcpy(&h.inv_y_bits, &c->inv_y, 4);
+  h.layer_hash = c->layer_hash;
   memcpy(hdr, &h, sizeof h);
   char* out = static_cast<char*>(dst);
   // the header is pageable host memory: the runtime stages it before cudaMemcpyAsync returns
@@ -2230,7 +3151,7 @@ int regtopk_state_import(regtopk_ctx* c, const void* src, size_t bytes) {
   memcpy(&mu_bits, &c->mu, 4);
   memcpy(&inv_y_bits, &c->inv_y, 4);
   if (h.magic != kStateMagic || h.d != c->d || h.k != c->k || h.N != c->N || h.ld != c->L.ld || h.W != c->L.W ||
-      h.grad_dtype != c->grad_dtype || h.mu_bits != mu_bits || h.inv_y_bits != inv_y_bits || h.round < 0 || (h.cur != 0 && h.cur != 1))
+      h.grad_dtype != c->grad_dtype || h.mu_bits != mu_bits || h.inv_y_bits != inv_y_bits || h.layer_hash != c->layer_hash || h.round < 0 || (h.cur != 0 && h.cur != 1))
     return REGTOPK_ERR_INVALID_ARG;
   rc = regtopk_state_reset(c);  // clears the control blocks and histograms as well
   if (!rc) rc = note_cuda(c, cudaMemcpyAsync(c->ws, in + kStateHeaderBytes, state_part1(c->L),

@@ -15,14 +15,15 @@ def bits(x):
 
 
 def run_parity(rounds, d, N, k, mu, omega=None, flags=0, check_eps=True, select_mode=0, threads=4,
-               reset_after=None, expect_dense=None, y=1.0, inplace=None):
+               reset_after=None, expect_dense=None, y=1.0, inplace=None, layers=None):
     """rounds: iterable of torch tensors [N, ld] (CPU or CUDA, float32 or bfloat16).
     inplace: None, or a function of the round number saying whether that round uses the accumulate-in-place calls.
+    layers: None, or (layer_end, layer_k) for one selection per layer (k is then ignored).
     Returns the library's stats after the last round."""
     rounds = iter(rounds)
     first = next(rounds)
-    lib = RegTopK(d, N, k, mu=mu, omega=omega, grad_dtype=first.dtype, flags=flags, y=y)
-    ora = OracleRegTopK(d, N, k, mu, omega=omega, select_mode=select_mode, threads=threads, y=y)
+    lib = RegTopK(d, N, k, mu=mu, omega=omega, grad_dtype=first.dtype, flags=flags, y=y, layers=layers)
+    ora = OracleRegTopK(d, N, k, mu, omega=omega, select_mode=select_mode, threads=threads, y=y, layers=layers)
     t = 0
     g = first
     while g is not None:

@@ -28,6 +28,16 @@ for (d, N, k) in [(1, 1, 1), (513, 3, 1), (4096, 8, 41), (65537, 2, 655), (20000
 stats.append(run_parity(gauss_rounds(3, 90_001, 4, seed=21), 90_001, 3, 900, 4.0, flags=DENSE, expect_dense=True))
 stats.append(run_parity(gauss_rounds(3, 90_001, 4, seed=21), 90_001, 3, 900, 4.0, flags=DENSE | WIDE, expect_dense=True))
 stats.append(run_parity(gauss_rounds(3, 150_000, 4, seed=8, quant=2), 150_000, 3, 1500, 4.0))
+GRID = binding.FLAG_GRID_DENSE_SELECT
+for (d, N, k) in [(1, 1, 1), (513, 3, 1), (16385, 2, 16385), (200003, 4, 2000), (2000, 1100, 20)]:
+    stats.append(run_parity(gauss_rounds(N, d, 3, seed=d + N), d, N, k, 4.0, flags=GRID | DENSE, expect_dense=True))
+stats.append(run_parity(gauss_rounds(3, 150_000, 4, seed=8, quant=2), 150_000, 3, 1500, 4.0, flags=GRID | DENSE))
+stats.append(run_parity([torch.full((2, 70_001), 0.5)] * 3, 70_001, 2, 700, 4.0, flags=GRID, expect_dense=True))
+import numpy as np
+sizes = [5000, 64, 64, 30_000, 128, 70_003, 3, 16385]
+layers = (np.cumsum(sizes).tolist(), [max(1, s // 50) for s in sizes])
+for fl in (0, WIDE):
+    stats.append(run_parity(gauss_rounds(3, sum(sizes), 4, seed=8, quant=2 if fl else 0), sum(sizes), 3, 0, 4.0, layers=layers, flags=fl))
 stats.append(run_parity(gauss_rounds(2, 120_007, 4, seed=12, ld=120_008, dtype=torch.bfloat16), 120_007, 2, 1200, 4.0))
 stats.append(run_parity(gauss_rounds(3, 100_001, 4, seed=9, ld=100_004), 100_001, 3, 1000, 4.0,
                         inplace=lambda t: t %% 2 == 1))

@@ -195,6 +195,106 @@ def test_sample_underestimates_cutoff():
     run_parity(rounds, d, N, k, 4.0, expect_dense=True)
 
 
+# ---- the dense exact path on the whole grid (what large problems and the layer-wise mode use), forced at small sizes ----
+GRID = binding.FLAG_GRID_DENSE_SELECT
+DENSE = binding.FLAG_FORCE_DENSE_SELECT
+
+
+@pytest.mark.parametrize("d,N,k", [(1, 1, 1), (7, 3, 7), (33, 2, 5), (513, 3, 1), (4096, 8, 41), (16384, 2, 100),
+                                   (16385, 2, 16385), (65537, 2, 655), (200003, 4, 2000), (1_000_003, 2, 10_000),
+                                   (3001, 33, 7), (2000, 1100, 20)])
+@pytest.mark.parametrize("mu", [4.0, 0.0])
+def test_grid_dense_sizes(d, N, k, mu):
+    run_parity(gauss_rounds(N, d, 4, seed=d + N + 2), d, N, k, mu, flags=GRID | DENSE, expect_dense=True, threads=8)
+
+
+def test_grid_dense_ties_zeros_bf16_wide_inplace():
+    d, N, k = 70_001, 2, 700
+    run_parity([torch.zeros(N, d) for _ in range(3)], d, N, k, 4.0, flags=GRID, expect_dense=True)
+    run_parity([torch.full((N, d), 0.5), torch.full((N, d), -0.25), torch.full((N, d), 0.5)], d, N, k, 4.0,
+               flags=GRID, expect_dense=True)
+    run_parity(gauss_rounds(3, 150_000, 4, seed=8, quant=2), 150_000, 3, 1500, 4.0, flags=GRID | DENSE)
+    run_parity(gauss_rounds(3, 150_000, 4, seed=8, quant=2), 150_000, 3, 1500, 4.0, flags=GRID | DENSE | WIDE)
+    run_parity(gauss_rounds(2, 100_001, 4, seed=10, ld=100_008, dtype=torch.bfloat16), 100_001, 2, 1000, 4.0,
+               flags=GRID | DENSE)
+    run_parity(gauss_rounds(3, 80_000, 4, seed=51), 80_000, 3, 800, 2.0, y=0.5, flags=GRID | DENSE,
+               inplace=lambda t: t % 2 == 0)
+
+
+def test_grid_dense_after_a_missed_cutoff():
+    """The sample's guess is too high for both workers (as in test_sample_overestimates_cutoff), with the flag that
+    hands such workers to the full-grid kernel; then a run in which only some rounds need it."""
+    d, N, k = 1_000_000, 2, 5000
+    pos = torch.from_numpy(_sample_positions(d))
+    rounds = []
+    for t, x in enumerate(gauss_rounds(N, d, 4, seed=30)):
+        if t != 2:
+            x[:, pos] *= 100.0
+        rounds.append(x)
+    run_parity(rounds, d, N, k, 4.0, flags=GRID, expect_dense=True)
+
+
+# ---- layer-wise selection: one Top-k per contiguous layer --------------------------------------------------
+def _layers_of(sizes, frac, kmin=1):
+    ends = np.cumsum(sizes).tolist()
+    ks = [int(min(s, max(kmin, int(frac * s + 0.5)))) for s in sizes]
+    return ends, ks
+
+
+@pytest.mark.parametrize("mu", [4.0, 0.0])
+def test_layerwise_tiny_and_ragged(mu):
+    for sizes, frac in [([1], 1.0), ([3, 4], 0.5), ([5, 1, 7, 2, 33], 0.3), ([64, 64, 1728, 64, 36864, 10], 0.05),
+                        ([16384, 16385, 3, 16383], 0.01), ([40_001, 7, 99_999], 0.02)]:
+        d = int(sum(sizes))
+        run_parity(gauss_rounds(3, d, 4, seed=d), d, 3, 0, mu, layers=_layers_of(sizes, frac))
+
+
+def test_layerwise_one_layer_is_the_global_selection():
+    d, N, k = 120_001, 3, 1200
+    rounds = list(gauss_rounds(N, d, 4, seed=77))
+    lib_l = RegTopK(d, N, k, mu=4.0, layers=([d], [k]))
+    lib_g = RegTopK(d, N, k, mu=4.0)
+    for g in rounds:
+        il, vl = lib_l.worker_step(g.cuda())
+        ig, vg = lib_g.worker_step(g.cuda())
+        assert torch.equal(il, ig) and torch.equal(vl.view(torch.int32), vg.view(torch.int32))
+        assert torch.equal(lib_l.aggregate().view(torch.int32), lib_g.aggregate().view(torch.int32))
+    lib_l.status(); lib_g.status()
+    run_parity(rounds, d, N, 0, 4.0, layers=([d], [k]))
+
+
+def test_layerwise_ties_zeros_bf16_wide_exponent():
+    sizes = [5000, 64, 64, 30_000, 128, 70_003]
+    d = int(sum(sizes))
+    L = _layers_of(sizes, 0.02)
+    run_parity(gauss_rounds(3, d, 4, seed=8, quant=2), d, 3, 0, 4.0, layers=L)
+    run_parity([torch.zeros(2, d) for _ in range(3)], d, 2, 0, 4.0, layers=L)
+    run_parity([torch.full((2, d), 0.5), torch.full((2, d), -0.25), torch.full((2, d), 0.5)], d, 2, 0, 4.0, layers=L)
+    run_parity(gauss_rounds(2, d, 4, seed=10, ld=d + 5, dtype=torch.bfloat16), d, 2, 0, 4.0, layers=L)
+    run_parity(gauss_rounds(3, d, 4, seed=11), d, 3, 0, 4.0, layers=L, flags=WIDE)
+    run_parity(gauss_rounds(3, d, 4, seed=12), d, 3, 0, 2.0, y=0.5, layers=L, inplace=lambda t: t % 2 == 1)
+    x = [g for g in gauss_rounds(2, d, 3, seed=13)]
+    for g in x:
+        g[:, 5000:5128] = 0.0  # two layers that are zero throughout: their winners are the lowest indices
+    run_parity(x, d, 2, 0, 4.0, layers=L)
+
+
+@pytest.mark.parametrize("name", ["resnet18", "resnet50", "gpt2"])
+def test_layerwise_scaled_workloads(name):
+    """The model-shaped tensor tables scaled down, every tensor a layer with the workload's sparsity."""
+    w = synth.workload(name, scale_to=300_000)
+    L = _layers_of(w.shapes, w.sparsity[-1])
+    s = synth.GradientStream(w, device="cpu", seed=19, pad_to=8)
+    run_parity((s.next() for _ in range(6)), w.d, w.N, 0, w.mu, layers=L)
+
+
+def test_layerwise_argument_errors():
+    for layers in [([10, 5], [1, 1]), ([5, 9], [1, 1]), ([5, 10], [0, 1]), ([5, 10], [6, 1]), ([5, 5, 10], [1, 1, 1])]:
+        with pytest.raises(RegTopKError):
+            RegTopK(10, 2, 2, layers=layers)
+    assert binding.workspace_bytes(10, 2, 3, layers=([5, 10], [1, 1])) == 0  # k must be the sum of the per-layer k
+
+
 # ---- the list handling of large N*k (separate full-grid kernels, pairs unzipped afterwards), forced at small
 #      sizes ------------------------------------------------------------------------------------------------
 WIDE = binding.FLAG_FORCE_WIDE_LISTS
