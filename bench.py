@@ -55,6 +55,10 @@ def parse():
     ap.add_argument("--select", default="global", choices=["global", "layerwise", "dense"],
                     help="layerwise: every tensor of the workload keeps its own share (one Top-k per layer); dense: the "
                          "exact full-grid selection from the rows is forced every round (the path a missed cutoff takes)")
+    ap.add_argument("--parallel", default="replicas", choices=["replicas", "by-worker"],
+                    help="by-worker: the workload's N workers are dealt to the ranks in contiguous blocks (N must be at least "
+                         "the number of ranks), one NCCL all-gather of the k pairs of every worker per round, every rank "
+                         "aggregates all N in worker order; total work is fixed as ranks are added (strong scaling)")
     ap.add_argument("--api", default="plain", choices=["plain", "inplace"],
                     help="inplace: the step is the caller's accumulate (torch add_ into the library's rows) + "
                          "regtopk_worker_step_inplace + regtopk_aggregate; the library's share is reported beside it")
@@ -363,6 +367,74 @@ def sweep_steps(w, arg):
     return int(max(10, min(1000, 300.0 / est_ms)))
 
 
+def run_by_worker(args, rank, world, local):
+    """The headline workload with its N workers spread over the ranks (paper_2501_05633_b200/sharded.py)."""
+    import copy
+    import torch
+    import torch.distributed as dist
+    import paper_2501_05633_b200 as pkg
+    from paper_2501_05633_b200 import synth
+    from paper_2501_05633_b200.sharded import ShardedRegTopK, worker_block
+    pkg.build()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29655")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    name, ki = (args.workload, args.sparsity_index or 0) if args.workload else HEADLINE
+    w = synth.workload(name)
+    k = w.k_values()[ki]
+    first, n_local = worker_block(w.N, rank, world)
+    wl = copy.deepcopy(w)
+    wl.N = n_local  # this rank generates its own block of the workers only (seeded per rank)
+    tdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+    stream = synth.GradientStream(wl, device=dev, seed=args.seed + 1000 * rank, pad_to=32)
+    bpe = 2 if w.grad_dtype == "bf16" else 4
+    per_batch = n_local * stream.ld * bpe
+    ring_n = int(max(2, min(args.ring or w.steps, (torch.cuda.mem_get_info()[0] * 0.45) // per_batch)))
+    ring = [stream.next() for _ in range(ring_n)]
+    lib = ShardedRegTopK(w.d, w.N, k, mu=w.mu, grad_dtype=tdt)
+    warmup = max(3, args.warmup)
+    for i in range(warmup):
+        lib.step(ring[i % ring_n])
+    lib.lib.status()
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.start()
+    l0 = lib.lib.stats()["kernel_launches"]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist.barrier(); torch.cuda.synchronize()
+    e0.record()
+    for i in range(args.steps):
+        lib.step(ring[(warmup + i) % ring_n])
+    e1.record()
+    dist.barrier(); torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    launches = lib.lib.stats()["kernel_launches"] - l0
+    lib.lib.status()
+    ms_all = max_over_ranks([ms], dev, world)[0]
+    if rank == 0:
+        coords = w.N * w.d
+        ms_step = ms_all / args.steps
+        alg_bytes = coords * (bpe + 8)
+        step_gbs = alg_bytes / (ms_step * 1e-3) / 1e9
+        peak, peak_kind = measured_peak()
+        line = {"metric": METRIC, "value": coords * args.steps / (ms_all * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
+                "scaling": "strong", "vs_baseline": None, "dtype": w.grad_dtype, "data": "synthetic",
+                "config": {"workload": workload_label(w, k, w.sparsity[ki]),
+                           "parallelism": f"workers sharded over {world} GPUs (blocks of {n_local} on rank 0), one NCCL "
+                                          f"all-gather of {8 * w.N * k} bytes of pairs per round, every rank aggregates all {w.N}",
+                           "l2": f"inputs larger than L2 ({per_batch / 1e6:.0f} MB per rank and step, ring of {ring_n} batches)",
+                           "step_hbm_gbs_all_ranks": step_gbs, "step_frac_of_measured_peak_per_gpu": step_gbs / peak / world,
+                           "peak_kind": f"of {peak_kind}"},
+                "clocks": clocks, "gpu_launches": launches}
+        print(json.dumps(line), flush=True)
+    dist.destroy_process_group()
+
+
 def main():
     args = parse()
     rank = int(os.environ.get("RANK", "0"))
@@ -370,6 +442,9 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+    if args.parallel == "by-worker":
+        run_by_worker(args, rank, world, local)
         return
     import torch
     import torch.distributed as dist

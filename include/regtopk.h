@@ -134,6 +134,23 @@ int regtopk_aggregate(regtopk_ctx* ctx, float* out_g);
  * Errors as regtopk_aggregate, plus INVALID_ARG for a non-finite eta. */
 int regtopk_aggregate_update(regtopk_ctx* ctx, float* theta, float eta, float* out_g);
 
+/* Server side of the round when the N workers are spread over several GPUs (one process and one context per GPU,
+ * each context holding a contiguous block of the workers; the paper's workers send their k pairs to a server,
+ * Section 2.2, and here every GPU plays the server for itself).  After regtopk_worker_step each process all-gathers
+ * the pairs of all workers (any transport; the data must be in this GPU's own memory, ordered by worker, before the
+ * call) and calls this instead of regtopk_aggregate: g^t = sum over all n_total workers of omega_n * ghat_n^t,
+ * added in the order n = 0..n_total-1 with each product rounded first, so that every GPU obtains the same g^t bit
+ * for bit; then the state roll.  g^t is what the next round's distortion (Eq. (Delta_def)) is formed from, which is
+ * why it must cover all workers and not only this context's.
+ *   all_idx, all_val  [n_total][k] pairs of all workers (device), this context's own among them.
+ *   omega_all         host array of n_total weights, or NULL for 1/n_total each.  The context itself must have been
+ *                     created with its own workers' weights out of the same array (its default of 1/N would be
+ *                     1/(workers of this context)).
+ *   out_g             [d] or NULL.
+ * Indices outside [0, d) are ignored.  Errors: INVALID_ARG, SEQUENCE (no worker_step since the last aggregate), CUDA. */
+int regtopk_aggregate_gathered(regtopk_ctx* ctx, int32_t n_total, const int32_t* all_idx, const float* all_val,
+                               const float* omega_all, float* out_g);
+
 /* Device pointer to the library's own copy of the latest aggregate g^t ([d] binary32, inside the
  * workspace, valid until the next regtopk_aggregate is enqueued).  *dev_ptr is written on the host. */
 int regtopk_global_gradient(regtopk_ctx* ctx, const float** dev_ptr);

@@ -28,6 +28,7 @@ EXPORTS = [
     "regtopk_get_stats", "regtopk_profile_enable", "regtopk_profile_read", "regtopk_debug_residual",
     "regtopk_destroy", "regtopk_strerror", "regtopk_aggregate_pairs_static", "regtopk_aggregate_update", "regtopk_state_bytes",
     "regtopk_state_export", "regtopk_state_import", "regtopk_accumulator", "regtopk_worker_step_inplace",
+    "regtopk_aggregate_gathered",
 ]
 
 
@@ -99,6 +100,8 @@ def load_library():
     L.regtopk_aggregate.argtypes = [vp, vp]
     L.regtopk_aggregate_update.restype = ctypes.c_int
     L.regtopk_aggregate_update.argtypes = [vp, vp, ctypes.c_float, vp]
+    L.regtopk_aggregate_gathered.restype = ctypes.c_int
+    L.regtopk_aggregate_gathered.argtypes = [vp, i32, vp, vp, ctypes.POINTER(ctypes.c_float), vp]
     L.regtopk_state_bytes.restype = ctypes.c_size_t
     L.regtopk_state_bytes.argtypes = [vp]
     L.regtopk_state_export.restype = ctypes.c_int
@@ -307,6 +310,25 @@ class RegTopK:
         _check(self.L.regtopk_aggregate_update(self.ctx, theta.data_ptr(), float(eta),
                                                out.data_ptr() if out is not None else None),
                "regtopk_aggregate_update")
+        return out if out is not None else self.global_gradient()
+
+    def aggregate_gathered(self, all_idx: torch.Tensor, all_val: torch.Tensor, omega_all=None,
+                           out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """aggregate() over the gathered pairs of all workers ([n_total, k] each, this context's own among them)
+        when the workers are spread over several contexts (regtopk_aggregate_gathered)."""
+        if not (all_idx.is_cuda and all_val.is_cuda and all_idx.dtype == torch.int32 and all_val.dtype == torch.float32
+                and all_idx.is_contiguous() and all_val.is_contiguous() and all_idx.shape == all_val.shape
+                and all_idx.dim() == 2 and all_idx.shape[1] == self.k):
+            raise TypeError("all_idx int32 and all_val float32 contiguous device tensors [n_total, k]")
+        n_total = int(all_idx.shape[0])
+        om = None
+        if omega_all is not None:
+            if len(omega_all) != n_total:
+                raise ValueError("omega_all needs one weight per gathered worker")
+            om = (ctypes.c_float * n_total)(*[float(x) for x in omega_all])
+        _check(self.L.regtopk_aggregate_gathered(self.ctx, n_total, all_idx.data_ptr(), all_val.data_ptr(), om,
+                                                 out.data_ptr() if out is not None else None),
+               "regtopk_aggregate_gathered")
         return out if out is not None else self.global_gradient()
 
     def state_export(self) -> torch.Tensor:

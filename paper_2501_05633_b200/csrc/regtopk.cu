@@ -2437,6 +2437,21 @@ __global__ void __launch_bounds__(256) k_aggregate(AggArgs p) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Aggregation over gathered pairs (regtopk_aggregate_gathered): the workers are spread over several GPUs, every GPU
+// has all workers' pairs after an all-gather and adds them into its own cleared g, one launch per worker in worker
+// order.  Within a worker the indices are distinct, so a launch has no two threads on one g[j], and the stream
+// orders the launches: g[j] = (((0 + w_0 v_0) + w_1 v_1) + ...) exactly as the server sum is defined.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_scatter_add(float* g, int64_t d, int64_t k, const int32_t* idx, const float* val,
+                                                     float omega) {
+  for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < k; r += (int64_t)gridDim.x * blockDim.x) {
+    const int32_t j = idx[r];
+    if ((u32)j >= (u32)d) continue;  // gathered data is not the library's own: an index out of range is ignored
+    g[j] = __fadd_rn(g[j], __fmul_rn(omega, val[r]));
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Aggregation from explicit pairs with built-in scratch (regtopk_aggregate_pairs_static).
 // The scratch is a file-scope device array: it costs 8 MiB on every GPU that loads this library,
 // and it is shared by all calls on that GPU.  Host code never uses the symbol as a pointer; it asks
@@ -3086,6 +3101,32 @@ int regtopk_aggregate_update(regtopk_ctx* c, float* theta, float eta, float* out
   if (out_g)
     rc = note_cuda(c, cudaMemcpyAsync(out_g, a.g, (size_t)c->d * 4, cudaMemcpyDeviceToDevice, c->stream));
   c->cur ^= 1;  // this round's pairs are now "previous"
+  c->round++;
+  c->stepped = 0;
+  return rc;
+}
+
+int regtopk_aggregate_gathered(regtopk_ctx* c, int32_t n_total, const int32_t* all_idx, const float* all_val,
+                               const float* omega_all, float* out_g) {
+  if (!c || n_total < 1 || n_total > 65535 || !all_idx || !all_val) return REGTOPK_ERR_INVALID_ARG;
+  if (omega_all)
+    for (int n = 0; n < n_total; ++n)
+      if (!isfinite(omega_all[n])) return REGTOPK_ERR_INVALID_ARG;
+  if (!c->stepped) return REGTOPK_ERR_SEQUENCE;
+  const Layout& L = c->L;
+  float* g = at<float>(c, L.off_g);
+  int rc = note_cuda(c, cudaMemsetAsync(g, 0, (size_t)c->d * 4, c->stream));
+  if (rc) return rc;
+  int64_t blocks = (c->k + 255) / 256;
+  if (blocks > (int64_t)c->num_sms * 16) blocks = (int64_t)c->num_sms * 16;
+  for (int n = 0; n < n_total; ++n) {
+    const float w = omega_all ? omega_all[n] : 1.0f / (float)n_total;
+    k_scatter_add<<<(unsigned)blocks, 256, 0, c->stream>>>(g, c->d, c->k, all_idx + (size_t)n * c->k,
+                                                           all_val + (size_t)n * c->k, w);
+    if ((rc = after_launch(c))) return rc;
+  }
+  if (out_g) rc = note_cuda(c, cudaMemcpyAsync(out_g, g, (size_t)c->d * 4, cudaMemcpyDeviceToDevice, c->stream));
+  c->cur ^= 1;  // this round's own pairs are now "previous"
   c->round++;
   c->stepped = 0;
   return rc;
