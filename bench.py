@@ -47,6 +47,9 @@ def parse():
                     help="time this workload only (no sweep); default: the headline workload plus the sweep")
     ap.add_argument("--sparsity-index", type=int, default=None)
     ap.add_argument("--ring", type=int, default=0, help="distinct gradient batches kept in HBM (0 = the workload's step count, capped by memory)")
+    ap.add_argument("--scale-to", type=int, default=0,
+                    help="with --workload: the same tensor table and value recipe scaled down to about this many "
+                         "coordinates (k scales with it); what the profiler captures of the larger shapes use")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--sweep-steps", type=int, default=0, help="timed steps per sweep variant (0 = chosen per workload, about 0.3 s each)")
     ap.add_argument("--no-sweep", action="store_true")
@@ -224,11 +227,11 @@ def run_reference(args, rank, world):
 class Bench:
     """One workload's gradient ring in HBM and the timing of its variants."""
 
-    def __init__(self, name, dev, seed, ring_arg, reserve_bytes=0):
+    def __init__(self, name, dev, seed, ring_arg, reserve_bytes=0, scale_to=0):
         import torch
         from paper_2501_05633_b200 import synth
         self.torch, self.dev = torch, dev
-        self.w = synth.workload(name)
+        self.w = synth.workload(name, scale_to=scale_to or None)
         self.bpe = 2 if self.w.grad_dtype == "bf16" else 4
         self.tdt = torch.bfloat16 if self.w.grad_dtype == "bf16" else torch.float32
         self.stream = synth.GradientStream(self.w, device=dev, seed=seed, pad_to=32)
@@ -500,7 +503,7 @@ def main():
                 del b
         head = b  # the headline workload's ring is the last one built
     else:
-        head = Bench(head_name, dev, args.seed + rank, args.ring)
+        head = Bench(head_name, dev, args.seed + rank, args.ring, scale_to=args.scale_to if single else 0)
 
     # ---- the headline: timed region with per-step events, clocks sampled meanwhile ----
     w = head.w

@@ -54,8 +54,10 @@ enum {
   REGTOPK_FLAG_FORCE_DENSE_SELECT = 2, /* testing: skip the sampled cutoff, always take the dense exact path */
   REGTOPK_FLAG_FORCE_WIDE_LISTS = 4,   /* testing: handle the candidate lists the way large N*k is handled (separate
                                           full-grid kernels, pairs unzipped afterwards) at any size; same results */
-  REGTOPK_FLAG_GRID_DENSE_SELECT = 8   /* testing: when a worker needs the dense exact path, run it as the full-grid
+  REGTOPK_FLAG_GRID_DENSE_SELECT = 8,  /* testing: when a worker needs the dense exact path, run it as the full-grid
                                           kernel that large problems use, at any size; same results              */
+  REGTOPK_FLAG_NUMERATORS_AT_AGGREGATE = 16 /* testing: form the numerators of the next round's distortion during the
+                                          aggregation, as is done for large d, at any size; same results          */
 };
 
 typedef struct {

@@ -21,6 +21,7 @@ _LIB = os.path.join(_PKG, "libregtopk.so")
 OK = 0
 GRAD_F32, GRAD_BF16 = 0, 1
 FLAG_HOST_STAGING, FLAG_FORCE_DENSE_SELECT, FLAG_FORCE_WIDE_LISTS, FLAG_GRID_DENSE_SELECT = 1, 2, 4, 8
+FLAG_NUMERATORS_AT_AGGREGATE = 16
 
 EXPORTS = [
     "regtopk_workspace_bytes", "regtopk_create", "regtopk_worker_step", "regtopk_aggregate",

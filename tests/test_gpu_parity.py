@@ -234,6 +234,29 @@ def test_grid_dense_after_a_missed_cutoff():
     run_parity(rounds, d, N, k, 4.0, flags=GRID, expect_dense=True)
 
 
+# ---- numerators of the distortion formed during the aggregation (what large d does), forced at small sizes ----
+def _shared_rounds(N, d, T, seed, dtype=torch.float32):
+    """Workers share most of their gradient, so that their masks overlap and one g[j] has many contributors."""
+    g = torch.Generator().manual_seed(seed)
+    for t in range(T):
+        base = torch.randn(d, generator=g)
+        yield (base[None, :] + 0.3 * torch.randn(N, d, generator=g)).to(dtype)
+
+
+def test_numerators_at_aggregate():
+    NUM = binding.FLAG_NUMERATORS_AT_AGGREGATE
+    for (d, N, k) in [(7, 3, 7), (4096, 8, 41), (200_003, 4, 2000), (70_000, 40, 700)]:
+        run_parity(_shared_rounds(N, d, 5, seed=d), d, N, k, 4.0, flags=NUM)
+    run_parity(_shared_rounds(5, 150_001, 5, seed=3), 150_001, 5, 1500, 2.0, flags=NUM | WIDE, omega=[0.1, 0.3, 0.2, 0.25, 0.15])
+    run_parity(_shared_rounds(4, 100_000, 5, seed=4, dtype=torch.bfloat16), 100_000, 4, 1000, 4.0, flags=NUM, y=0.5,
+               inplace=lambda t: t % 2 == 1)
+    run_parity(_shared_rounds(3, 90_001, 5, seed=5), 90_001, 3, 900, 4.0, flags=NUM | DENSE | GRID)
+    # rounds with and without the numerators mixed: a reset and a state import fall back to the gather from g
+    d, N, k = 60_000, 3, 600
+    rounds = list(_shared_rounds(N, d, 6, seed=6))
+    run_parity(rounds, d, N, k, 4.0, flags=NUM, reset_after=3)
+
+
 # ---- layer-wise selection: one Top-k per contiguous layer --------------------------------------------------
 def _layers_of(sizes, frac, kmin=1):
     ends = np.cumsum(sizes).tolist()
