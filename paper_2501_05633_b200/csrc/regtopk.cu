@@ -1554,10 +1554,11 @@ __global__ void __launch_bounds__(256) k_unzip(UnzipArgs p) {
 //
 // Per segment:
 //   (A) a histogram of the top 12 key bits over the segment's part of the row, restricted to keys at or above
-//       a lower bound `lo` (a hint: the sampled cutoff, or last round's threshold lowered by an octave), so
+//       a lower bound `lo` (a hint: the sampled cutoff, or the bin edge near last round's 3 k_s-th largest key), so
 //       that nearly all entries cost a compare and no shared-memory atomic.  From the top down, the bin b0 that
 //       holds the k_s-th largest, the entries above it and the number c0 inside it.  If the histogram holds
-//       fewer than k_s entries the hint was too high and the pass is repeated for that segment with lo = 0.
+//       fewer than k_s entries the hint was too high and the pass is repeated for that segment with lo an octave
+//       lower, and if need be a third time with lo = 0.
 //   (B) a second pass over the rows: entries above bin b0 are winners (mask bit set, composite appended to
 //       the worker's winner list); the c0 entries inside it go to a list of their own,
 //   (C) from which one block takes the `need` largest composites (key, lowest index).
@@ -1576,8 +1577,8 @@ constexpr int kDenseMaxFlagged = 1024;
 constexpr u32 kOctave = 0x00800000u;  // one binary order of magnitude in key units
 constexpr u32 kHintMargin = 2u << 19;  // two bins of the first digit (an eighth of an octave)
 
-enum : u32 { kSegList = 0u, kSegRows = 1u, kSegRetry = 2u };
-enum : u32 { kFlagRetry = 1u, kFlagRows = 2u, kFlagOrdered = 4u, kFlagBad = 8u };
+enum : u32 { kSegList = 0u, kSegRows = 1u, kSegRetry = 2u, kSegList2 = 3u };
+enum : u32 { kFlagRetry = 1u, kFlagRows = 2u, kFlagOrdered = 4u, kFlagBad = 8u, kFlagRows2 = 16u };
 
 struct __align__(16) SegState {
   u32 prefix;  // digits of the threshold key fixed so far
@@ -1587,7 +1588,7 @@ struct __align__(16) SegState {
   u32 lo;      // keys below this are left out of the first histogram
   u32 boff;    // kSegList: where the segment's in-bin list starts in the worker's B list
   u32 bfill;   //           entries written there so far
-  u32 pad;
+  u32 sh;      // key bits below the digits in `prefix` (19 after the first digit, 7 after the second)
 };
 
 struct DenseArgs {
@@ -1603,7 +1604,7 @@ struct DenseArgs {
   const int64_t* seg_tile0; // [n_seg + 1] first tile of each segment
   u32* dhist;               // [N][n_seg][kBins], all zero between launches
   SegState* seg;            // [N][n_seg]
-  u32* seg_thr;             // [N][n_seg] a lower bound of the segment's threshold key in the last round it came here (0: none)
+  u32* seg_thr;             // [N][n_seg] the lower bound the last round left for this one (a bin edge near its 3k-th largest key; 0: none)
   u32* tile_ties;           // [N][tiles][2]: entries equal to the threshold key in the tile, and in lower tiles of the segment
 };
 
@@ -1694,8 +1695,24 @@ __device__ __forceinline__ SegState load_seg(const DenseArgs& a, int n, int s) {
   const uint4 v = __ldcg(q), x = __ldcg(q + 1);
   SegState r;
   r.prefix = v.x; r.need = v.y; r.ties = v.z; r.mode = v.w;
-  r.lo = x.x; r.boff = x.y; r.bfill = x.z; r.pad = x.w;
+  r.lo = x.x; r.boff = x.y; r.bfill = x.z; r.sh = x.w;
   return r;
+}
+
+// Take `want` entries of a list of `cap` whose fill counter is *fill, but only if they fit: the counter never
+// passes cap, so space that was granted is never granted twice.  One thread; at most a few retries under contention.
+__device__ __forceinline__ bool reserve_list_space(u32* fill, u32 want, u64 cap, u32* off) {
+  u32 cur = *reinterpret_cast<volatile u32*>(fill);
+  for (int tries = 0; tries < 1024; ++tries) {
+    if ((u64)cur + want > cap) return false;
+    const u32 seen = atomicCAS(fill, cur, cur + want);
+    if (seen == cur) {
+      *off = cur;
+      return true;
+    }
+    cur = seen;
+  }
+  return false;  // (gives up: the segment then takes the way that needs no list)
 }
 
 // The tile `w` of the run of tiles the flagged workers have together: worker, segment and index range.
@@ -1915,7 +1932,14 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         const u32 need = lv ? old.need : (u32)(a.seg_kpre[s + 1] - a.seg_kpre[s]);
         __syncthreads();
         block_find_from_top(s_hist, kBins, need, s_scan, s_res);
-        if (tid == 0) done(n, s, old, need, s_res[0], s_res[1], s_res[0] == kFull ? 0u : s_hist[s_res[0]]);
+        const u32 b = s_res[0], above = s_res[1];
+        u32 b_wide = kFull;  // first digit only: the bin of the entry three times as far down, for the next round's bound
+        if (lv == 0 && b != kFull) {
+          __syncthreads();
+          block_find_from_top(s_hist, kBins, 3u * need, s_scan, s_res);
+          b_wide = s_res[0];
+        }
+        if (tid == 0) done(n, s, old, need, b, above, b == kFull ? 0u : s_hist[b], b_wide);
         __syncthreads();
       }
     };
@@ -1925,8 +1949,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
       u32 lo;
       if (a.layered) {
-        const u32 thr = a.seg_thr[(size_t)n * a.n_seg + s];  // lower edge of the bin of last round's threshold
-        lo = thr > kHintMargin ? thr - kHintMargin : 0u;
+        lo = a.seg_thr[(size_t)n * a.n_seg + s];  // left by the last round (0: none)
       } else {
         // the sampled cutoff as it is when the path was asked for; an octave lower when that cutoff has just left
         // too few entries above it
@@ -1934,23 +1957,23 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         lo = hint == kFull ? 0u : (p.ctl[n].force_dense ? hint : (hint > kOctave ? hint - kOctave : 0u));
       }
       SegState st;
-      st.prefix = 0; st.need = 0; st.ties = 0; st.mode = kSegRetry; st.lo = lo; st.boff = 0; st.bfill = 0; st.pad = 0;
+      st.prefix = 0; st.need = 0; st.ties = 0; st.mode = kSegRetry; st.lo = lo; st.boff = 0; st.bfill = 0; st.sh = 19;
       a.seg[(size_t)n * a.n_seg + s] = st;
     }
     grid.sync();
 
-    // ---- (A) first digit; once more with lo = 0 for the segments whose hint was too high ----
-    for (int attempt = 0; attempt < 2; ++attempt) {
+    // ---- (A) first digit; again with lo an octave lower, then with lo = 0, for the segments whose hint was too high ----
+    for (int attempt = 0; attempt < 3; ++attempt) {
       hist_pass(0, kSegRetry);
       grid.sync();
-      find_pass(0, kSegRetry, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin) {
+      find_pass(0, kSegRetry, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin, u32 b_wide) {
         SegState* st = a.seg + (size_t)n * a.n_seg + s;
         if (b == kFull) {
           if (old.lo == 0u) {  // fewer than k entries in the whole segment: cannot happen
             atomicOr(&p.gctl->dense_flags, kFlagBad);
             st->mode = kSegList; st->prefix = 0; st->need = 0; st->ties = 0;
-          } else {
-            st->lo = 0u;  // stays kSegRetry
+          } else {  // stays kSegRetry: first an octave lower, then without a bound
+            st->lo = (attempt == 0 && old.lo > kOctave) ? old.lo - kOctave : 0u;
             atomicOr(&p.gctl->dense_flags, kFlagRetry);
           }
           return;
@@ -1958,10 +1981,18 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         st->prefix = b;
         st->need = need - above;
         st->ties = in_bin;
-        a.seg_thr[(size_t)n * a.n_seg + s] = b << 19;  // lower edge of the bin: next round's hint
+        // next round's lower bound: the lower edge of the bin that holds this round's 3k-th largest entry; if fewer
+        // than that were counted, two bins below this round's bound
+        // (but at least one whole bin below the threshold's own: the bins are 1/16 octave wide)
+        {
+          const u32 below = b > 0u ? b - 1u : 0u;
+          const u32 edge = b_wide != kFull ? (b_wide < below ? b_wide : below) << 19
+                                           : (old.lo > kHintMargin ? old.lo - kHintMargin : 0u);
+          a.seg_thr[(size_t)n * a.n_seg + s] = edge;
+        }
         // room for the bin's entries in the worker's B list?
-        const u32 off = atomicAdd(&p.ctl[n].bcount, in_bin);
-        if ((u64)off + in_bin <= (u64)p.stride) {
+        u32 off;
+        if (reserve_list_space(&p.ctl[n].bcount, in_bin, (u64)p.stride, &off)) {
           st->mode = kSegList;
           st->boff = off;
         } else {
@@ -1976,7 +2007,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
     }
 
     // ---- (B) second pass over the rows: winners above the bin, and the bin's own entries to their list ----
-    {
+    auto compact_pass = [&](u32 want_mode) {
       int cur_n = -1, cur_s = -1;
       // During the walk a thread that holds an entry at or above the bin's lower edge puts it into its warp's
       // staging list itself (one shared-memory counter).  When the list is half full, or the segment changes, the
@@ -1988,7 +2019,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         return p.use_marks && ((__ldg(p.mask_old + (size_t)n * p.W + (j >> 5)) >> (j & 31)) & 1u);
       };
       auto place = [&](int n, int s, const SegState& sg, u64 c, bool live) {  // all lanes of the warp; live: this lane has an entry
-        const bool isA = live && (u32)(c >> 51) > sg.prefix;  // key >> 19
+        const bool isA = live && (u32)(c >> (32u + sg.sh)) > sg.prefix;  // the key's digits fixed so far
         const bool isB = live && !isA;
         const u32 mA = __ballot_sync(kFull, isA), mB = __ballot_sync(kFull, isB);
         u32 baseA = 0, baseB = 0;
@@ -2022,7 +2053,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       auto direct = [&](int n, int s, const SegState& sg, u64 c) {
         const u32 j = composite_idx(c);
         if (marked(n, j)) return;
-        if ((u32)(c >> 51) > sg.prefix) {
+        if ((u32)(c >> (32u + sg.sh)) > sg.prefix) {
           set_winner(p.mask_new + (size_t)n * p.W, j, p.d);
           const u32 pos = atomicAdd(&p.ctl[n].acount, 1u);
           if (RT_INB(pos < k)) p.candA[(size_t)n * p.stride + pos] = c;
@@ -2038,12 +2069,12 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       for (int64_t w = w_begin; w < w_end; ++w) {
         const DenseTile t = dense_tile(a, s_flagged, w);
         if (t.n != cur_n || t.s != cur_s) {
-          if (cur_n >= 0 && st.mode == kSegList) flush(cur_n, cur_s, st);
+          if (cur_n >= 0 && st.mode == want_mode) flush(cur_n, cur_s, st);
           cur_n = t.n; cur_s = t.s;
           st = load_seg(a, t.n, t.s);  // but for its fill counter, nothing writes it during this pass
         }
-        if (st.mode != kSegList) continue;  // the same in every thread of the block
-        const u32 floor_key = max(st.prefix << 19, st.lo);  // nothing below it is a winner or in the bin
+        if (st.mode != want_mode) continue;  // the same in every thread of the block
+        const u32 floor_key = max(st.prefix << st.sh, st.lo);  // nothing below it is a winner or in the bin
         dense_walk<true, true>(p, t.n, t.t0, t.t1, floor_key,
           [&](int64_t j4, const u32 (&key)[4], const bool (&in)[4]) {
 #pragma unroll
@@ -2059,7 +2090,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             if (*reinterpret_cast<volatile u32*>(&s_wcnt[0][warp]) >= kCap / 2u) flush(t.n, t.s, st);
           });
       }
-      if (cur_n >= 0 && st.mode == kSegList) flush(cur_n, cur_s, st);
+      if (cur_n >= 0 && st.mode == want_mode) flush(cur_n, cur_s, st);
       u32 cntA = 0;  // from here on the lists are filled by ballot: warp-uniform fill
       auto flush_A2 = [&](int n) {
         stage_flush(listA, cntA, &p.ctl[n].acount, p.candA + (size_t)n * p.stride, (u64)k, lane);
@@ -2081,9 +2112,9 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             st.boff = 0; st.ties = 0;
             if (live) {
               st = load_seg(a, n, s);
-              if (st.mode == kSegList) {
-                win = (key >> 19) > st.prefix;
-                bin = (key >> 19) == st.prefix && key >= st.lo;
+              if (st.mode == want_mode) {
+                win = (key >> st.sh) > st.prefix;
+                bin = (key >> st.sh) == st.prefix && key >= st.lo;
               }
             }
             const u64 c = make_composite(key, (u32)j);
@@ -2100,16 +2131,18 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
           flush_A2(n);
         }
       }
-    }
+    };
+    compact_pass(kSegList);
     const u32 flags0 = __ldcg(&p.gctl->dense_flags);  // written before the last barrier
     if (flags0 & kFlagRows) hist_pass(1, kSegRows);
     grid.sync();
 
     // ---- (C) per list segment: the `need` largest composites of its in-bin list win ----
-    for (int64_t v = blockIdx.x; v < nsegs; v += gridDim.x) {
+    auto list_select = [&](u32 want_mode) {
+     for (int64_t v = blockIdx.x; v < nsegs; v += gridDim.x) {
       const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
       const SegState st = load_seg(a, n, s);
-      if (st.mode != kSegList || st.need == 0u) continue;  // the same in every thread of the block
+      if (st.mode != want_mode || st.need == 0u) continue;  // the same in every thread of the block
       const u64* list = p.candB + (size_t)n * p.stride + st.boff;
       u32* mask = p.mask_new + (size_t)n * p.W;
       const u32 count = st.ties;
@@ -2161,19 +2194,37 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         }
         carry += total;
       }
-    }
+     }
+    };
+    list_select(kSegList);
     if (flags0 & kFlagRows) {
-      find_pass(1, kSegRows, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin) {
+      // Second digit of the segments whose first bin was too crowded for the list space.  After it the bin is 4096
+      // times narrower: if it fits now, the segment goes the list way from here (one more pass over the rows);
+      // otherwise (rows of equal keys) the third digit and the ordered take of ties follow.
+      find_pass(1, kSegRows, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin, u32) {
         SegState* st = a.seg + (size_t)n * a.n_seg + s;
         if (b == kFull) { atomicOr(&p.gctl->dense_flags, kFlagBad); b = 0; above = 0; }
         st->prefix = (old.prefix << 12) | b;
         st->need = need - above;
         st->ties = in_bin;
+        st->sh = 7;
+        u32 off;
+        if (reserve_list_space(&p.ctl[n].bcount, in_bin, (u64)p.stride, &off)) {
+          st->mode = kSegList2;
+          st->boff = off;
+          st->lo = 0u;  // the second digit counted every entry with the first digit's prefix
+        } else {
+          atomicOr(&p.gctl->dense_flags, kFlagRows2);
+        }
       });
       grid.sync();
-      hist_pass(2, kSegRows);
+      const u32 flags_b = __ldcg(&p.gctl->dense_flags);
+      compact_pass(kSegList2);
+      if (flags_b & kFlagRows2) hist_pass(2, kSegRows);
       grid.sync();
-      find_pass(2, kSegRows, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin) {
+      list_select(kSegList2);
+     if (flags_b & kFlagRows2) {
+      find_pass(2, kSegRows, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin, u32) {
         SegState* st = a.seg + (size_t)n * a.n_seg + s;
         if (b == kFull) { atomicOr(&p.gctl->dense_flags, kFlagBad); b = 0; above = 0; }
         st->prefix = (old.prefix << 7) | b;
@@ -2283,6 +2334,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         }
         if (cur_n >= 0) flush_A(cur_n);
       }
+     }
     }
     grid.sync();
     // every flagged worker must have gathered exactly k winners
