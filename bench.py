@@ -85,9 +85,11 @@ def stream_section_hash():
     return hashlib.sha256(src[a:b].encode()).hexdigest()
 
 
-def recorded_traffic(workload_name, grad_dtype, api):
-    """DRAM bytes of one k_stream launch from the profiler capture summarised under profiles/, or None when there is
-    no capture for this workload or the kernel's source has changed since it was taken."""
+def recorded_traffic(workload_name, grad_dtype, api, coords):
+    """DRAM bytes of one k_stream launch over `coords` coordinates, from the profiler capture summarised under
+    profiles/ (taken on the same workload scaled down where the full size is too large to capture: the kernel's
+    traffic is proportional to the coordinates it streams, so the capture's bytes per coordinate are scaled up), or
+    None when there is no capture for this workload or the kernel's source has changed since it was taken."""
     try:
         rec = json.load(open(os.path.join(ROOT, "profiles", "k_stream_traffic.json")))
     except Exception:
@@ -96,7 +98,7 @@ def recorded_traffic(workload_name, grad_dtype, api):
     for r in rec.get("captures", []):
         if (r.get("workload") == workload_name and r.get("grad_dtype") == grad_dtype and r.get("api", "plain") == api
                 and now is not None and r.get("stream_section_sha256") == now):
-            return r.get("dram_bytes_per_launch")
+            return r["dram_bytes_per_launch"] / r["coordinates_per_launch"] * coords
     return None
 
 
@@ -573,7 +575,7 @@ def main():
             "gpu_launches": r["launches"],
             "roofline": {"bound": "hbm", "kernel": "k_stream", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                         "traffic": recorded_traffic(w.name, w.grad_dtype, args.api),
+                         "traffic": recorded_traffic(w.name, w.grad_dtype, args.api, coords),
                          "algorithmic_bytes_per_launch": r["kern_alg_bytes"], "avg_launch_ms": r["kern_avg_ms"]},
         }
         if inplace:

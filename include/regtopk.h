@@ -182,6 +182,9 @@ int regtopk_round_host(regtopk_ctx* ctx, const void* h_grads, int64_t grad_ld, i
 
 /* Synchronises the stream and returns REGTOPK_OK or the sticky error recorded by the device
  * (REGTOPK_ERR_INTERNAL) or by CUDA (REGTOPK_ERR_CUDA); a device error survives regtopk_state_reset.
+ * REGTOPK_ERR_INTERNAL means that a consistency check of the selection failed (a bug in the library): the round in
+ * which it happened may have left pairs, masks and residuals that do not belong together, so the state is to be
+ * discarded (regtopk_state_reset, or import of an earlier export); the code stays set so that it cannot go unnoticed.
  * The checked build of the library (-DREGTOPK_DEBUG=1) also returns REGTOPK_ERR_INVALID_ARG here once an
  * accumulator was infinite or NaN (gradients must be finite), until the next regtopk_state_reset. */
 int regtopk_status(regtopk_ctx* ctx);
