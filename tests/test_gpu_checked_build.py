@@ -33,6 +33,17 @@ for (d, N, k) in [(1, 1, 1), (513, 3, 1), (16385, 2, 16385), (200003, 4, 2000), 
     stats.append(run_parity(gauss_rounds(N, d, 3, seed=d + N), d, N, k, 4.0, flags=GRID | DENSE, expect_dense=True))
 stats.append(run_parity(gauss_rounds(3, 150_000, 4, seed=8, quant=2), 150_000, 3, 1500, 4.0, flags=GRID | DENSE))
 stats.append(run_parity([torch.full((2, 70_001), 0.5)] * 3, 70_001, 2, 700, 4.0, flags=GRID, expect_dense=True))
+# a threshold bin too crowded for the list space (second digit, then the list), and a block of equal magnitudes at
+# the threshold (third digit, ordered ties)
+gen = torch.Generator().manual_seed(77)
+for ties in (False, True):
+    crowded = []
+    for t in range(3):
+        x = (1.0 + 0.04 * torch.rand(3, 300_000, generator=gen)) * torch.where(torch.rand(3, 300_000, generator=gen) < 0.5, -1.0, 1.0)
+        if ties:
+            x[:, 1000:60_000] = 1.042
+        crowded.append(x)
+    stats.append(run_parity(crowded, 300_000, 3, 3000, 4.0, flags=GRID | DENSE, expect_dense=True))
 import numpy as np
 sizes = [5000, 64, 64, 30_000, 128, 70_003, 3, 16385]
 layers = (np.cumsum(sizes).tolist(), [max(1, s // 50) for s in sizes])

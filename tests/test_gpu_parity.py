@@ -221,6 +221,29 @@ def test_grid_dense_ties_zeros_bf16_wide_inplace():
                inplace=lambda t: t % 2 == 0)
 
 
+def test_grid_dense_crowded_threshold_bin():
+    """Most of a row inside one bin of the first digit (magnitudes within 4 % of each other, all different): the bin
+    does not fit the list space, the second digit narrows it until it does.  Then the same with a block of exactly
+    equal magnitudes around the threshold, which needs the third digit and the ordered take of ties."""
+    d, N, k = 300_000, 3, 3000
+    g = torch.Generator().manual_seed(77)
+
+    def rounds(ties):
+        out = []
+        for t in range(4):
+            x = (1.0 + 0.04 * torch.rand(N, d, generator=g)) * torch.where(torch.rand(N, d, generator=g) < 0.5, -1.0, 1.0)
+            x[:, ::7] *= 1e-3  # a share of small entries
+            if ties:
+                x[:, 1000:60_000] = 1.042  # 59,000 equal magnitudes above all others: the threshold falls among them
+            out.append(x)
+        return out
+
+    for ties in (False, True):
+        run_parity(rounds(ties), d, N, k, 4.0, flags=GRID | DENSE, expect_dense=True)
+        run_parity(rounds(ties), d, N, 0, 4.0, layers=([100_000, 100_064, 300_000], [1000, 7, 1993]))
+        run_parity(rounds(ties), d, N, k, 0.0, flags=GRID | DENSE | WIDE, expect_dense=True)
+
+
 def test_grid_dense_after_a_missed_cutoff():
     """The sample's guess is too high for both workers (as in test_sample_overestimates_cutoff), with the flag that
     hands such workers to the full-grid kernel; then a run in which only some rounds need it."""
