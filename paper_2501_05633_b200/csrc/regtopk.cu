@@ -1562,10 +1562,12 @@ __global__ void __launch_bounds__(256) k_unzip(UnzipArgs p) {
 //   (B) a second pass over the rows: entries above bin b0 are winners (mask bit set, composite appended to
 //       the worker's winner list); the c0 entries inside it go to a list of their own,
 //   (C) from which one block takes the `need` largest composites (key, lowest index).
-// A segment whose bin b0 does not fit the list space (rows full of equal values) stays on the rows instead:
-// two more digits of 12 and 7 bits give the threshold key T and the number of entries equal to T that are
-// to be taken; if there are more of those than needed, their counts per tile are scanned so that the lowest
-// indices win; a last pass over the rows sets the winners.
+// A segment whose bin b0 does not fit the list space (error feedback has packed thousands of entries into it, or
+// the row is full of equal values) stays on the rows for a second digit of 12 bits.  If its bin, 4096 times
+// narrower, fits, the segment goes the list way from there ((B) and (C) with 24 bits fixed).  Otherwise a third
+// digit of 7 bits gives the threshold key T and the number of entries equal to T that are to be taken; if there
+// are more of those than needed, their counts per tile are scanned so that the lowest indices win; a last pass
+// over the rows sets the winners.
 // Rows are cut into tiles of kDenseTile coordinates that never straddle a segment; a block owns a
 // contiguous run of tiles.  If nobody needs the path the kernel returns at once.
 // ---------------------------------------------------------------------------------------------
