@@ -64,6 +64,7 @@ constexpr int kBlockSel = 1024;            // threads per block of k_sample_cuto
 constexpr int kBlockPost = REGTOPK_POST_THREADS;  // threads per block of k_post
 constexpr int kStreamThreads = 256;
 constexpr int kWarpList = 256;             // per-warp staging list of k_stream (entries)
+constexpr int kCutSpan = 512;              // coordinates per entry of the layer-wise cutoff table (divides every chunk size)
 constexpr int kBins = 4096;                // histogram bins of the select
 constexpr int kMaxCluster = 16;
 constexpr int kMaxSegments = kMaxCluster * 32;  // mask segments per row: one per warp of a k_post cluster
@@ -607,6 +608,8 @@ struct StreamArgs {
   int64_t stride;
   const u32* marks;  // [N][W] last round's mask, or NULL: entries on it are not candidates (their
   int64_t W;         // regularised score comes from the override list instead)
+  const u32* chunk_cut;  // layer-wise mode: [N][cuts] candidate cutoff per kCutSpan coordinates (the layers have
+  int64_t cuts;          // their own thresholds), instead of one per worker; else NULL
 };
 
 // Write a warp's staged hits to the worker's candidate list.  With a previous mask, the entries on it
@@ -731,6 +734,13 @@ __global__ void __launch_bounds__(kStreamThreads, StreamShape<BF16, VEC, INPLACE
       marks = p.marks ? p.marks + (size_t)n * p.W : nullptr;
     }
     const bool full = base + S::kChunk <= p.d;  // warp-uniform
+    if (p.chunk_cut) {  // layer-wise: the lowest cutoff of the layers this chunk meets (admits a superset)
+      const u32* cc = p.chunk_cut + (size_t)n * p.cuts + base / kCutSpan;
+      cutoff = __ldg(cc);
+#pragma unroll
+      for (int i = 1; i < S::kChunk / kCutSpan; ++i)
+        if (base + (int64_t)i * kCutSpan < p.d) cutoff = min(cutoff, __ldg(cc + i));
+    }
     float4 e[S::kSteps][S::kVec], g[S::kSteps][S::kVec];
 #pragma unroll
     for (int u = 0; u < S::kSteps; ++u) {
@@ -1137,6 +1147,7 @@ __device__ __forceinline__ void post_emit(const PostArgs& p, int n, u32 first_t,
   const u32* qpre = p.qprefix + (size_t)n * (p.W >> 2);
   const u32 nA = took_dense ? k : ncand;
   const u32 total_items = nA + (took_dense ? 0u : novr);
+  if (took_dense) A = O;  // every flavour of the dense path leaves its k winners in the override-composite row
   for (u32 t0 = first_t; t0 < total_items; t0 += 4 * stride_t) {
     u64 c[4];
     uint4 qw[4];
@@ -1312,6 +1323,7 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
   } else {
     // ---- exact selection over the whole row: three radix digits of the 31-bit key ----
     took_dense = true;
+    u64* Wl = p.ovr_comp + (size_t)n * p.k;  // the winners' list (the row is free on this path: see post_emit)
     if (rk == 0 && tid == 0) atomicAdd(&p.gctl->dense_workers, 1ull);
     // this block's part of the row; the cuts are multiples of four so that every thread reads whole quads
     const int64_t c0 = (int64_t)(((u64)rk * (u64)p.d) / CS) & ~(int64_t)3;
@@ -1358,7 +1370,7 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
         const bool gt = j4 + q < c1 && key[q] > T;
         my_ties += (j4 + q < c1 && key[q] == T) ? 1u : 0u;
         const u32 pos = warp_reserve_global(gt, &ctl->acount);
-        if (gt && pos < n_gt) A[pos] = make_composite(key[q], (u32)(j4 + q));
+        if (gt && pos < n_gt) Wl[pos] = make_composite(key[q], (u32)(j4 + q));
       }
     }
     u32 block_ties;
@@ -1385,7 +1397,7 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         if (j4 + q < c1 && key[q] == T) {
-          if (rank < need && RT_INB(n_gt + rank < k)) A[n_gt + rank] = make_composite(T, (u32)(j4 + q));
+          if (rank < need && RT_INB(n_gt + rank < k)) Wl[n_gt + rank] = make_composite(T, (u32)(j4 + q));
           ++rank;
         }
       }
@@ -1394,7 +1406,7 @@ __global__ void __launch_bounds__(kBlockPost, 1024 / kBlockPost) k_post(PostArgs
     cl.sync();  // winner list complete
     if (rk == 0 && tid == 0 && (bad || __ldcg(&ctl->acount) != n_gt)) atomicOr(&p.gctl->err, kErrDenseSelect);
     if (!bad)
-      for (u32 i = first_t; i < k; i += stride_t) set_winner(mask, composite_idx(__ldcg(&A[i])), p.d);
+      for (u32 i = first_t; i < k; i += stride_t) set_winner(mask, composite_idx(__ldcg(&Wl[i])), p.d);
     cl.sync();  // every winner bit is set
   }
   if (p.wide) {  // k_wide_prefix and k_wide_emit take over
@@ -1591,6 +1603,9 @@ struct __align__(16) SegState {
   u32 boff;    // kSegList: where the segment's in-bin list starts in the worker's B list
   u32 bfill;   //           entries written there so far
   u32 sh;      // key bits below the digits in `prefix` (19 after the first digit, 7 after the second)
+  u32 src;     // 1: the first digit and the compaction read the worker's candidate list (layer-wise mode: the streaming
+               //    pass gathered every entry at or above the segment's bound); 0: they walk the rows
+  u32 pad[3];
 };
 
 struct DenseArgs {
@@ -1692,12 +1707,37 @@ __device__ __forceinline__ int dense_seg_of_index(const int64_t* seg_end, int n_
   return lo;
 }
 
+// Layer-wise mode, before the streaming pass: the candidate cutoff of every span of kCutSpan coordinates, i.e. the
+// lowest of the bounds that the last round left for the layers the span meets (seg_thr; a layer without one admits
+// nothing, 0xFFFFFFFF, and is selected from the rows).  The streaming pass then compacts, per worker, every entry that
+// can matter to its layer, and k_dense takes the layers' first histogram and their winners from that list instead
+// of from two more passes over the rows.
+__global__ void __launch_bounds__(256) k_layer_cutoffs(u32* chunk_cut, int64_t cuts, int64_t d, int N, int n_seg,
+                                                       const int64_t* seg_end, const u32* seg_thr) {
+  grid_dependency_begin();
+  const int64_t total = cuts * N;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int n = (int)(i / cuts);
+    const int64_t c = i - (int64_t)n * cuts;
+    const int64_t j0 = c * kCutSpan, j1 = j0 + kCutSpan < d ? j0 + kCutSpan : d;
+    u32 cut = kFull;
+    for (int s = dense_seg_of_index(seg_end, n_seg, j0); s < n_seg; ++s) {
+      const u32 thr = seg_thr[(size_t)n * n_seg + s];
+      const u32 lo = thr ? thr : kFull;
+      cut = lo < cut ? lo : cut;
+      if (seg_end[s] >= j1) break;
+    }
+    chunk_cut[i] = cut;
+  }
+}
+
 __device__ __forceinline__ SegState load_seg(const DenseArgs& a, int n, int s) {  // written by other blocks of this launch
   const uint4* q = reinterpret_cast<const uint4*>(a.seg + (size_t)n * a.n_seg + s);
-  const uint4 v = __ldcg(q), x = __ldcg(q + 1);
+  const uint4 v = __ldcg(q), x = __ldcg(q + 1), y = __ldcg(q + 2);
   SegState r;
   r.prefix = v.x; r.need = v.y; r.ties = v.z; r.mode = v.w;
   r.lo = x.x; r.boff = x.y; r.bfill = x.z; r.sh = x.w;
+  r.src = y.x; r.pad[0] = r.pad[1] = r.pad[2] = 0u;
   return r;
 }
 
@@ -1787,6 +1827,9 @@ __device__ __forceinline__ void stage_flush(u64* list, u32& count, u32* fill, u6
   __syncwarp();
 }
 
+// LAYERED: layer-wise mode (hints from last round's segments, segments fed from the candidate list); the plain
+// instance carries none of that code.
+template <bool LAYERED>
 __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
   extern __shared__ __align__(16) u64 s_stage[];  // [kDenseWarps][2 * kWarpList]: per-warp staging lists
   __shared__ __align__(16) u32 s_hist[kBins];
@@ -1852,7 +1895,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
           cur_n = t.n; cur_s = t.s;
           st = load_seg(a, t.n, t.s);  // nothing writes it during this pass
         }
-        if (st.mode != want_mode) continue;  // the same in every thread of the block
+        if (st.mode != want_mode || (LAYERED && lv == 0 && st.src)) { w += a.seg_tile0[t.s + 1] - 1 - t.t; continue; }  // nothing to do in this segment: on to its last tile (the same in every thread of the block)
         dirty = true;
         const u32 floor_key = lv == 0 ? st.lo : st.prefix << (shf + width);  // no entry below it is counted
         auto count = [&](int64_t j4, const u32 (&key)[4], const bool (&in)[4]) {
@@ -1878,6 +1921,32 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       }
       __syncthreads();
       if (dirty) flush_hist(s_hist, a.dhist + ((size_t)cur_n * a.n_seg + cur_s) * kBins, kBins);
+      if (LAYERED && lv == 0) {
+        // segments fed from the candidate list: one lane per entry, straight into the segments' histograms
+        for (int64_t f = 0; f < nf; ++f) {
+          const int n = (int)s_flagged[f];
+          const u32 cc = p.ctl[n].cand_count;
+          if ((u64)cc > (u64)p.capA) continue;  // overflowed: no segment of this worker is list-fed
+          const u64* cand = p.candA + (size_t)n * p.stride;
+          for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + (tid & ~31); i0 < (int64_t)cc; i0 += (int64_t)gridDim.x * blockDim.x) {
+            const int64_t i = i0 + lane;
+            bool use = i < (int64_t)cc;
+            const u64 c = use ? __ldcg(&cand[i]) : 0ull;
+            const u32 key = (u32)(c >> 32);
+            const int s = (use && a.n_seg > 1) ? dense_seg_of_index(a.seg_end, a.n_seg, (int64_t)composite_idx(c)) : 0;
+            if (use) {
+              const SegState st = load_seg(a, n, s);
+              use = st.mode == want_mode && st.src && key >= st.lo;
+            }
+            u32* target = a.dhist + ((size_t)n * a.n_seg + s) * kBins + (key >> 19);
+            const u32 act = __ballot_sync(kFull, use);
+            if (use) {
+              const u32 peers = __match_any_sync(act, (u64)(uintptr_t)target);
+              if (lane == __ffs(peers) - 1) atomicAdd(target, (u32)__popc(peers));
+            }
+          }
+        }
+      }
       if (lv == 0 && p.use_marks) {
         // the entries of the previous support, which the walk above left out: their scores come from the override
         // list (index order), one lane per entry, straight into the segments' histograms in global memory
@@ -1895,9 +1964,9 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             u32 lo_seg = 0;
             if (use) {
               const SegState st = load_seg(a, n, s);
-              take_back = st.mode == want_mode;
+              take_back = st.mode == want_mode && !(LAYERED && st.src);  // (a list-fed segment never counted it: the list has no such entries)
               lo_seg = st.lo;
-              use = take_back && key >= st.lo;
+              use = st.mode == want_mode && key >= st.lo;
             }
             u32* hist = a.dhist + ((size_t)n * a.n_seg + s) * kBins;
             u32* target = hist + (key >> 19);
@@ -1950,7 +2019,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
     for (int64_t v = (int64_t)blockIdx.x * blockDim.x + tid; v < nsegs; v += (int64_t)gridDim.x * blockDim.x) {
       const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
       u32 lo;
-      if (a.layered) {
+      if (LAYERED) {
         lo = a.seg_thr[(size_t)n * a.n_seg + s];  // left by the last round (0: none)
       } else {
         // the sampled cutoff as it is when the path was asked for; an octave lower when that cutoff has just left
@@ -1960,6 +2029,10 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       }
       SegState st;
       st.prefix = 0; st.need = 0; st.ties = 0; st.mode = kSegRetry; st.lo = lo; st.boff = 0; st.bfill = 0; st.sh = 19;
+      // layer-wise: the candidate list holds every entry of the segment at or above lo, unless there was no bound to
+      // gather by or the list overflowed
+      st.src = (LAYERED && lo != 0u && (u64)p.ctl[n].cand_count <= (u64)p.capA) ? 1u : 0u;
+      st.pad[0] = st.pad[1] = st.pad[2] = 0u;
       a.seg[(size_t)n * a.n_seg + s] = st;
     }
     grid.sync();
@@ -1974,7 +2047,8 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
           if (old.lo == 0u) {  // fewer than k entries in the whole segment: cannot happen
             atomicOr(&p.gctl->dense_flags, kFlagBad);
             st->mode = kSegList; st->prefix = 0; st->need = 0; st->ties = 0;
-          } else {  // stays kSegRetry: first an octave lower, then without a bound
+          } else {  // stays kSegRetry: first an octave lower, then without a bound; from the rows in any case
+            st->src = 0u;
             st->lo = (attempt == 0 && old.lo > kOctave) ? old.lo - kOctave : 0u;
             atomicOr(&p.gctl->dense_flags, kFlagRetry);
           }
@@ -2033,7 +2107,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         if (isA) {
           set_winner(p.mask_new + (size_t)n * p.W, composite_idx(c), p.d);
           const u32 pos = baseA + __popc(mA & lt);
-          if (RT_INB(pos < k)) p.candA[(size_t)n * p.stride + pos] = c;
+          if (RT_INB(pos < k)) p.ovr_comp[(size_t)n * p.k + pos] = c;
         }
         if (isB) {
           const u32 pos = baseB + __popc(mB & lt);
@@ -2058,7 +2132,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         if ((u32)(c >> (32u + sg.sh)) > sg.prefix) {
           set_winner(p.mask_new + (size_t)n * p.W, j, p.d);
           const u32 pos = atomicAdd(&p.ctl[n].acount, 1u);
-          if (RT_INB(pos < k)) p.candA[(size_t)n * p.stride + pos] = c;
+          if (RT_INB(pos < k)) p.ovr_comp[(size_t)n * p.k + pos] = c;
         } else {
           const u32 pos = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, 1u);
           if (RT_INB(pos < sg.ties)) p.candB[(size_t)n * p.stride + sg.boff + pos] = c;
@@ -2075,7 +2149,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
           cur_n = t.n; cur_s = t.s;
           st = load_seg(a, t.n, t.s);  // but for its fill counter, nothing writes it during this pass
         }
-        if (st.mode != want_mode) continue;  // the same in every thread of the block
+        if (st.mode != want_mode || (LAYERED && want_mode == kSegList && st.src)) { w += a.seg_tile0[t.s + 1] - 1 - t.t; continue; }  // nothing to do in this segment: on to its last tile (the same in every thread of the block)
         const u32 floor_key = max(st.prefix << st.sh, st.lo);  // nothing below it is a winner or in the bin
         dense_walk<true, true>(p, t.n, t.t0, t.t1, floor_key,
           [&](int64_t j4, const u32 (&key)[4], const bool (&in)[4]) {
@@ -2095,8 +2169,44 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       if (cur_n >= 0 && st.mode == want_mode) flush(cur_n, cur_s, st);
       u32 cntA = 0;  // from here on the lists are filled by ballot: warp-uniform fill
       auto flush_A2 = [&](int n) {
-        stage_flush(listA, cntA, &p.ctl[n].acount, p.candA + (size_t)n * p.stride, (u64)k, lane);
+        stage_flush(listA, cntA, &p.ctl[n].acount, p.ovr_comp + (size_t)n * p.k, (u64)k, lane);
       };
+      if (LAYERED && want_mode == kSegList) {  // the segments fed from the candidate list
+        for (int64_t f = 0; f < nf; ++f) {
+          const int n = (int)s_flagged[f];
+          const u32 cc = p.ctl[n].cand_count;
+          if ((u64)cc > (u64)p.capA) continue;
+          const u64* cand = p.candA + (size_t)n * p.stride;
+          u32* mask = p.mask_new + (size_t)n * p.W;
+          for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + (tid & ~31); i0 < (int64_t)cc; i0 += (int64_t)gridDim.x * blockDim.x) {
+            const int64_t i = i0 + lane;
+            const bool live = i < (int64_t)cc;
+            const u64 c = live ? __ldcg(&cand[i]) : 0ull;
+            const u32 key = (u32)(c >> 32), j = composite_idx(c);
+            const int s = (live && a.n_seg > 1) ? dense_seg_of_index(a.seg_end, a.n_seg, (int64_t)j) : 0;
+            bool win = false, bin = false;
+            SegState st;
+            st.boff = 0; st.ties = 0;
+            if (live) {
+              st = load_seg(a, n, s);
+              if (st.mode == kSegList && st.src) {
+                win = (key >> st.sh) > st.prefix;
+                bin = (key >> st.sh) == st.prefix && key >= st.lo;
+              }
+            }
+            if (win) set_winner(mask, j, p.d);
+            if (bin) {
+              const u32 pos = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, 1u);
+              if (RT_INB(pos < st.ties)) p.candB[(size_t)n * p.stride + st.boff + pos] = c;
+            }
+            if (__any_sync(kFull, win)) {
+              stage_add(listA, cntA, win, c, lane);
+              if (cntA >= (u32)(kWarpList - 32)) flush_A2(n);
+            }
+          }
+          flush_A2(n);
+        }
+      }
       if (p.use_marks) {  // the same for the entries of the previous support, from the override list
         for (int64_t f = 0; f < nf; ++f) {
           const int n = (int)s_flagged[f];
@@ -2182,7 +2292,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       if (tid == 0) s_cnt = atomicAdd(&p.ctl[n].acount, st.need);
       __syncthreads();
       const u32 abase = s_cnt;
-      u64* A = p.candA + (size_t)n * p.stride;
+      u64* A = p.ovr_comp + (size_t)n * p.k;
       u32 carry = 0;
       for (u32 i0 = 0; i0 < count; i0 += blockDim.x) {
         const u32 i = i0 + tid;
@@ -2243,7 +2353,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         for (int64_t w = w_begin; w < w_end; ++w) {
           const DenseTile t = dense_tile(a, s_flagged, w);
           const SegState st = load_seg(a, t.n, t.s);
-          if (st.mode != kSegRows || st.ties <= st.need) continue;  // the same in every thread of the block
+          if (st.mode != kSegRows || st.ties <= st.need) { w += a.seg_tile0[t.s + 1] - 1 - t.t; continue; }  // nothing to do in this segment: on to its last tile (the same in every thread of the block)
           if (tid == 0) s_cnt = 0;
           __syncthreads();
           u32 mine = 0;
@@ -2281,7 +2391,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         u32 cntA = 0;
         int cur_n = -1;
         auto flush_A = [&](int n) {
-          stage_flush(listA, cntA, &p.ctl[n].acount, p.candA + (size_t)n * p.stride, (u64)k, lane);
+          stage_flush(listA, cntA, &p.ctl[n].acount, p.ovr_comp + (size_t)n * p.k, (u64)k, lane);
         };
         for (int64_t w = w_begin; w < w_end; ++w) {
           const DenseTile t = dense_tile(a, s_flagged, w);
@@ -2290,7 +2400,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             cur_n = t.n;
           }
           const SegState st = load_seg(a, t.n, t.s);
-          if (st.mode != kSegRows) continue;  // the same in every thread of the block
+          if (st.mode != kSegRows) { w += a.seg_tile0[t.s + 1] - 1 - t.t; continue; }  // nothing to do in this segment: on to its last tile (the same in every thread of the block)
           const u32 T = st.prefix, need = st.need;
           // all of the tile's ties win, none of them, or (one tile per segment at most) the first few in index order
           bool all_win = st.ties <= need, none_win = false;
@@ -2622,6 +2732,8 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 struct Layout {
   int64_t ld, W, capA, stride;
   int64_t n_seg, tiles;  // segments of a row (layers; 1 in the plain mode) and k_dense tiles per row
+  int64_t cuts;          // entries per row of the layer-wise cutoff table
+  size_t off_chunk_cut;
   size_t off_dhist, off_seg_thr, off_seg, off_tile_ties, off_seg_end, off_seg_kpre, off_seg_tile0;
   size_t off_eps, off_g, off_mask[2], off_ctl, off_gctl, off_shist, zero_end, off_skeys, off_qprefix, off_segtot, off_segbase, off_ghist, off_btot, off_idx[2], off_val[2],
       off_ovr_key, off_ovr_comp, off_candA, off_candB, off_num[2], off_omega, off_stage_g, off_stage_idx,
@@ -2677,6 +2789,9 @@ Layout make_layout(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
   const int64_t M = d < kSampleMax ? d : kSampleMax;
   const int64_t kt = pr->mu > 0.0f ? (2 * k < d ? 2 * k : d) : k;
   int64_t cap = 3 * kt + 64 * ((d + M - 1) / M) + 4096;
+  // layer-wise mode gathers by per-layer bounds that are a coarse bin edge below each layer's threshold: room for
+  // many times k (measured 17-22 k on the ResNet-18 tensor table)
+  if (pr->n_layers > 0 && cap < 48 * k + 4096) cap = 48 * k + 4096;
   if (cap > d) cap = d;
   if (cap < k) cap = k;
   L.capA = cap;
@@ -2701,6 +2816,8 @@ Layout make_layout(int64_t d, int32_t N, int64_t k, const regtopk_params* pr) {
   L.off_seg_end = take((size_t)L.n_seg * 8);
   L.off_seg_kpre = take((size_t)(L.n_seg + 1) * 8);
   L.off_seg_tile0 = take((size_t)(L.n_seg + 1) * 8);
+  L.cuts = (d + kCutSpan - 1) / kCutSpan;
+  L.off_chunk_cut = take(pr->n_layers > 0 ? (size_t)N * L.cuts * 4 : 0);
   L.off_skeys = take((size_t)N * kSampleMax * 4);
   L.off_qprefix = take((size_t)N * (L.W / 4) * 4);
   L.off_segtot = take((size_t)N * kMaxSegments * 4);
@@ -2942,8 +3059,9 @@ int regtopk_create(regtopk_ctx** out, int64_t d, int32_t N, int64_t k, const reg
                    d * (int64_t)N >= kGridDenseCoords) ? 1 : 0;
   {
     int per_sm = 0;
-    if (cudaFuncSetAttribute(k_dense, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dense_smem()) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_dense, kDenseThreads, dense_smem()) != cudaSuccess ||
+    const void* dense_fn = c->layered ? (const void*)k_dense<true> : (const void*)k_dense<false>;
+    if (cudaFuncSetAttribute(dense_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dense_smem()) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dense_fn, kDenseThreads, dense_smem()) != cudaSuccess ||
         per_sm < 1) {
       cudaGetLastError();
       per_sm = 1;
@@ -3041,6 +3159,18 @@ int step_impl(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_i
   st.grads = grads; st.grad_ld = grad_ld; st.eps = at<float>(c, L.off_eps); st.ld = L.ld; st.d = c->d;
   st.N = c->N; st.ctl = sa.ctl; st.cand = at<u64>(c, L.off_candA); st.cap = L.capA; st.stride = L.stride;
   st.marks = use_marks ? at<u32>(c, L.off_mask[prev]) : nullptr; st.W = L.W;
+  st.chunk_cut = nullptr; st.cuts = L.cuts;
+  if (c->layered) {
+    st.chunk_cut = at<u32>(c, L.off_chunk_cut);
+    int64_t blocks = (L.cuts * c->N + 255) / 256;
+    if (blocks > (int64_t)c->num_sms * 8) blocks = (int64_t)c->num_sms * 8;
+    cudaLaunchConfig_t lcfg;
+    cudaLaunchAttribute lattr[2];
+    launch_config(&lcfg, lattr, (unsigned)blocks, 1, 256, 0, c->stream);
+    cudaLaunchKernelEx(&lcfg, k_layer_cutoffs, at<u32>(c, L.off_chunk_cut), L.cuts, c->d, (int)c->N, (int)L.n_seg,
+                       (const int64_t*)at<int64_t>(c, L.off_seg_end), (const u32*)at<u32>(c, L.off_seg_thr));
+    if ((rc = after_launch(c))) return rc;
+  }
   const bool prof = c->profiling && c->n_events < kMaxProfile;
   if (prof) cudaEventRecord(c->ev0[c->n_events], c->stream);
   if (inplace) launch_stream<false, true, true>(c, st, 4);
@@ -3110,7 +3240,7 @@ int step_impl(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_i
     dattr[0].val.cooperative = 1;
     dcfg.attrs = dattr;
     dcfg.numAttrs = 1;
-    cudaError_t de = cudaLaunchKernelEx(&dcfg, k_dense, da);
+    cudaError_t de = c->layered ? cudaLaunchKernelEx(&dcfg, k_dense<true>, da) : cudaLaunchKernelEx(&dcfg, k_dense<false>, da);
     c->launches++;
     if (de != cudaSuccess) return note_cuda(c, de);
     if ((rc = note_cuda(c, cudaGetLastError()))) return rc;
