@@ -2195,9 +2195,17 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
               }
             }
             if (win) set_winner(mask, j, p.d);
-            if (bin) {
-              const u32 pos = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, 1u);
-              if (RT_INB(pos < st.ties)) p.candB[(size_t)n * p.stride + st.boff + pos] = c;
+            {  // the bin's entries to their segment's list: lanes of one segment reserve their places together
+              const u32 act = __ballot_sync(kFull, bin);
+              if (bin) {
+                const u32 peers = __match_any_sync(act, (u32)s);
+                const int leader = __ffs(peers) - 1;
+                u32 base = 0;
+                if (lane == leader) base = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, (u32)__popc(peers));
+                base = __shfl_sync(peers, base, leader);
+                const u32 pos = base + (u32)__popc(peers & ((1u << lane) - 1u));
+                if (RT_INB(pos < st.ties)) p.candB[(size_t)n * p.stride + st.boff + pos] = c;
+              }
             }
             if (__any_sync(kFull, win)) {
               stage_add(listA, cntA, win, c, lane);
@@ -2231,9 +2239,17 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             }
             const u64 c = make_composite(key, (u32)j);
             if (win) set_winner(mask, (u32)j, p.d);
-            if (bin) {
-              const u32 pos = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, 1u);
-              if (RT_INB(pos < st.ties)) p.candB[(size_t)n * p.stride + st.boff + pos] = c;
+            {  // the bin's entries to their segment's list: lanes of one segment reserve their places together
+              const u32 act = __ballot_sync(kFull, bin);
+              if (bin) {
+                const u32 peers = __match_any_sync(act, (u32)s);
+                const int leader = __ffs(peers) - 1;
+                u32 base = 0;
+                if (lane == leader) base = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, (u32)__popc(peers));
+                base = __shfl_sync(peers, base, leader);
+                const u32 pos = base + (u32)__popc(peers & ((1u << lane) - 1u));
+                if (RT_INB(pos < st.ties)) p.candB[(size_t)n * p.stride + st.boff + pos] = c;
+              }
             }
             if (__any_sync(kFull, win)) {
               stage_add(listA, cntA, win, c, lane);
@@ -2260,6 +2276,26 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       const u32 count = st.ties;
       if (st.bfill != count) {
         if (tid == 0) atomicOr(&p.gctl->dense_flags, kFlagBad);
+        continue;
+      }
+      if (count <= blockDim.x) {
+        // a short list (the usual case): every thread ranks its entry against all others in shared memory; the
+        // entry with `above` larger ones before it takes place `above` among the segment's winners from this list
+        u64* items = reinterpret_cast<u64*>(s_hist);
+        __syncthreads();
+        const u64 mine = (u32)tid < count ? __ldcg(&list[tid]) : 0ull;
+        if ((u32)tid < count) items[tid] = mine;
+        if (tid == 0) s_cnt = atomicAdd(&p.ctl[n].acount, st.need);
+        __syncthreads();
+        if ((u32)tid < count) {
+          u32 above = 0;
+          for (u32 j = 0; j < count; ++j) above += items[j] > mine ? 1u : 0u;
+          if (above < st.need) {
+            set_winner(mask, composite_idx(mine), p.d);
+            if (RT_INB((u64)s_cnt + above < (u64)k)) p.ovr_comp[(size_t)n * p.k + s_cnt + above] = mine;
+          }
+        }
+        __syncthreads();
         continue;
       }
       // the need-th largest composite, byte by byte (the list stays where it is)
