@@ -118,7 +118,8 @@ struct WorkerCtl {
                     // across rounds (nothing else resets it but regtopk_state_reset)
   u32 exact_window; // length of the last such stretch: it doubles with every further fallback
   u32 hint;         // the sampled cutoff of this round, kept for k_dense when the candidate path is not taken (0xFFFFFFFF: none)
-  u32 pad[2];
+  u32 seg_done;     // k_dense: segments of this worker whose first digit has been searched in the current pass; zero between passes
+  u32 pad;
 };
 
 struct GlobalCtl {
@@ -1591,8 +1592,10 @@ constexpr int kDenseMaxFlagged = 1024;
 constexpr u32 kOctave = 0x00800000u;  // one binary order of magnitude in key units
 constexpr u32 kHintMargin = 2u << 19;  // two bins of the first digit (an eighth of an octave)
 
-enum : u32 { kSegList = 0u, kSegRows = 1u, kSegRetry = 2u, kSegList2 = 3u };
-enum : u32 { kFlagRetry = 1u, kFlagRows = 2u, kFlagOrdered = 4u, kFlagBad = 8u, kFlagRows2 = 16u };
+enum : u32 { kSegList = 0u, kSegRows = 1u, kSegRetry = 2u, kSegList2 = 3u,
+             kSegWant = 4u };  // first digit found, list space not yet dealt out (only inside the first-digit search)
+enum : u32 { kFlagRetry = 1u, kFlagRows = 2u, kFlagOrdered = 4u, kFlagBad = 8u, kFlagRows2 = 16u,
+            kFlagWalk = 32u };  // layer-wise mode: some segment takes its first digit from the rows (otherwise no block walks its tiles for it)
 
 struct __align__(16) SegState {
   u32 prefix;  // digits of the threshold key fixed so far
@@ -1834,9 +1837,11 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
   extern __shared__ __align__(16) u64 s_stage[];  // [kDenseWarps][2 * kWarpList]: per-warp staging lists
   __shared__ __align__(16) u32 s_hist[kBins];
   __shared__ u32 s_flagged[kDenseMaxFlagged];
+  __shared__ u32 s_cbase[kDenseMaxFlagged + 1];  // layer-wise mode: 32-entry pieces of the candidate lists before each flagged worker's
   __shared__ u32 s_scan[33];
-  __shared__ u32 s_res[3];
-  __shared__ u32 s_cnt, s_nf;
+  __shared__ u32 s_res[4];
+  __shared__ u32 s_cnt, s_nf, s_nf2;
+  __shared__ u64 s_T;
   __shared__ u32 s_wcnt[1][kDenseWarps];
   cg::grid_group grid = cg::this_grid();
   const PostArgs& p = a.p;
@@ -1868,10 +1873,30 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
     const int64_t w_begin = (int64_t)blockIdx.x * per < total_tiles ? (int64_t)blockIdx.x * per : total_tiles;
     const int64_t w_end = w_begin + per < total_tiles ? w_begin + per : total_tiles;
     const int64_t nsegs = nf * a.n_seg;
+    if (LAYERED) {  // (a worker whose list overflowed has no pieces: none of its segments is fed from the list)
+      constexpr int kPer = kDenseMaxFlagged / kDenseThreads;
+      u32 mine[kPer], sum = 0, total;
+#pragma unroll
+      for (int i = 0; i < kPer; ++i) {
+        const int64_t f = kPer * tid + i;
+        u32 cc = 0;
+        if (f < nf) cc = p.ctl[s_flagged[f]].cand_count;
+        mine[i] = (u64)cc <= (u64)p.capA ? (cc + 31u) >> 5 : 0u;
+        sum += mine[i];
+      }
+      u32 at = block_excl_scan(sum, s_scan, &total);
+#pragma unroll
+      for (int i = 0; i < kPer; ++i) {
+        s_cbase[kPer * tid + i] = at;
+        at += mine[i];
+      }
+      if (tid == 0) s_cbase[kDenseMaxFlagged] = total;
+      __syncthreads();
+    }
 
     // One histogram pass over this block's tiles.  which(seg state) says whether a segment takes part; the entries
     // counted are those with key >= lo (first digit) or whose higher digits equal the prefix (later digits).
-    auto hist_pass = [&](int lv, u32 want_mode) {
+    auto hist_pass = [&](int lv, u32 want_mode, bool walk) {
       const int shf = lv == 0 ? 19 : (lv == 1 ? 7 : 0);  // digits of 12, 12 and 7 bits
       const int width = lv == 2 ? 7 : 12;
       const u32 nbm = (1u << width) - 1u;
@@ -1881,7 +1906,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       st.mode = ~0u;
       for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
       __syncthreads();
-      for (int64_t w = w_begin; w < w_end; ++w) {
+      for (int64_t w = walk ? w_begin : w_end; w < w_end; ++w) {
         const DenseTile t = dense_tile(a, s_flagged, w);
         if (t.n != cur_n || t.s != cur_s) {
           if (dirty) {
@@ -1922,22 +1947,71 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       __syncthreads();
       if (dirty) flush_hist(s_hist, a.dhist + ((size_t)cur_n * a.n_seg + cur_s) * kBins, kBins);
       if (LAYERED && lv == 0) {
-        // segments fed from the candidate list: one lane per entry, straight into the segments' histograms
-        for (int64_t f = 0; f < nf; ++f) {
-          const int n = (int)s_flagged[f];
-          const u32 cc = p.ctl[n].cand_count;
-          if ((u64)cc > (u64)p.capA) continue;  // overflowed: no segment of this worker is list-fed
-          const u64* cand = p.candA + (size_t)n * p.stride;
-          for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + (tid & ~31); i0 < (int64_t)cc; i0 += (int64_t)gridDim.x * blockDim.x) {
-            const int64_t i = i0 + lane;
-            bool use = i < (int64_t)cc;
-            const u64 c = use ? __ldcg(&cand[i]) : 0ull;
-            const u32 key = (u32)(c >> 32);
-            const int s = (use && a.n_seg > 1) ? dense_seg_of_index(a.seg_end, a.n_seg, (int64_t)composite_idx(c)) : 0;
-            if (use) {
-              const SegState st = load_seg(a, n, s);
-              use = st.mode == want_mode && st.src && key >= st.lo;
+        // Layer-wise mode: the candidate lists of the segments fed from them, and the entries of the previous
+        // support (override list), as one run of 32-entry tasks over all flagged workers, dealt to the warps of the
+        // grid in contiguous pieces.  The segment ends and the segments' bounds are looked up in shared memory
+        // (the staging space, not used in this pass) when they fit there.
+        u32* t_end = reinterpret_cast<u32*>(s_stage);  // [n_seg]
+        u32* t_lo = t_end + a.n_seg;                   // [nsegs]: bound | list-fed, or kFull if the segment takes no part
+        const bool fast = (u64)nsegs + (u64)a.n_seg <= (u64)kDenseWarps * 2u * kWarpList * 2u;
+        if (fast) {
+          for (int i = tid; i < a.n_seg; i += blockDim.x) t_end[i] = (u32)a.seg_end[i];
+          for (int64_t v = tid; v < nsegs; v += blockDim.x) {
+            const SegState sg = load_seg(a, (int)s_flagged[v / a.n_seg], (int)(v % a.n_seg));
+            t_lo[v] = sg.mode == want_mode ? (sg.lo | sg.src) : kFull;
+          }
+          __syncthreads();
+        }
+        auto seg_of = [&](u32 j) -> int {
+          if (!fast) return dense_seg_of_index(a.seg_end, a.n_seg, (int64_t)j);
+          int lo = 0, hi = a.n_seg - 1;  // the first segment whose end lies beyond j
+          while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (t_end[mid] <= j) lo = mid + 1; else hi = mid;
+          }
+          return lo;
+        };
+        auto bound_of = [&](int64_t f, int n, int s) -> u32 {
+          if (fast) return t_lo[f * a.n_seg + s];
+          const SegState sg = load_seg(a, n, s);
+          return sg.mode == want_mode ? (sg.lo | sg.src) : kFull;
+        };
+        const int64_t gw = (int64_t)blockIdx.x * kDenseWarps + warp, nwarps = (int64_t)gridDim.x * kDenseWarps;
+        {  // candidates
+          const int64_t tasks = s_cbase[nf];
+          const int64_t per = (tasks + nwarps - 1) / nwarps;
+          const int64_t t0 = gw * per, t1 = t0 + per < tasks ? t0 + per : tasks;
+          int64_t f = 0;
+          if (t0 < t1) {
+            int64_t lo = 0, hi = nf;  // the worker whose tasks include t0
+            while (hi - lo > 1) {
+              const int64_t mid = (lo + hi) >> 1;
+              if ((int64_t)s_cbase[mid] <= t0) lo = mid; else hi = mid;
             }
+            f = lo;
+          }
+          auto fetch = [&](int64_t t, int64_t& ff, bool& live) -> u64 {
+            live = false;
+            if (t >= t1) return 0ull;
+            while (t >= (int64_t)s_cbase[ff + 1]) ++ff;
+            const int n = (int)s_flagged[ff];
+            const int64_t i = (t - (int64_t)s_cbase[ff]) * 32 + lane;
+            live = i < (int64_t)p.ctl[n].cand_count;
+            return live ? __ldcg(p.candA + (size_t)n * p.stride + i) : 0ull;
+          };
+          int64_t f_next = f;
+          bool live_next = false;
+          u64 c_next = fetch(t0, f_next, live_next);
+          for (int64_t t = t0; t < t1; ++t) {
+            const u64 c = c_next;
+            const bool live = live_next;
+            f = f_next;
+            c_next = fetch(t + 1, f_next, live_next);
+            const int n = (int)s_flagged[f];
+            const u32 key = (u32)(c >> 32);
+            const int s = (live && a.n_seg > 1) ? seg_of(composite_idx(c)) : 0;
+            const u32 bound = live ? bound_of(f, n, s) : kFull;
+            const bool use = bound != kFull && (bound & 1u) && key >= (bound & ~1u);
             u32* target = a.dhist + ((size_t)n * a.n_seg + s) * kBins + (key >> 19);
             const u32 act = __ballot_sync(kFull, use);
             if (use) {
@@ -1946,7 +2020,38 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             }
           }
         }
-      }
+        if (p.use_marks) {  // the previous support: scores from the override list (index order)
+          const int64_t per_w = (p.k + 31) / 32, tasks = nf * per_w;
+          const int64_t per = (tasks + nwarps - 1) / nwarps;
+          const int64_t t0 = gw * per, t1 = t0 + per < tasks ? t0 + per : tasks;
+          for (int64_t t = t0; t < t1; ++t) {
+            const int64_t f = t / per_w;
+            const int n = (int)s_flagged[f];
+            const int64_t i = (t - f * per_w) * 32 + lane;
+            const bool live = i < p.k;
+            const int32_t j = live ? p.prev_idx[(size_t)n * p.k + i] : 0;
+            const u32 key = live ? __ldcg(&p.ovr_key[(size_t)n * p.k + i]) : 0u;
+            const int s = (live && a.n_seg > 1) ? seg_of((u32)j) : 0;
+            const u32 bound = live ? bound_of(f, n, s) : kFull;
+            const bool part = bound != kFull;
+            const u32 lo_seg = bound & ~1u;
+            const bool use = part && key >= lo_seg;
+            u32* hist = a.dhist + ((size_t)n * a.n_seg + s) * kBins;
+            u32* target = hist + (key >> 19);
+            const u32 act = __ballot_sync(kFull, use);
+            if (use) {  // lanes that count into the same bin add once
+              const u32 peers = __match_any_sync(act, (u64)(uintptr_t)target);
+              if (lane == __ffs(peers) - 1) atomicAdd(target, (u32)__popc(peers));
+            }
+            // a segment counted from the rows has the entry under bits(|a|): take that back (a list-fed one never
+            // counted it: the list has no entries of the previous support)
+            if (part && !(bound & 1u)) {
+              const u32 ka = __float_as_uint(p.eps[(size_t)n * p.ld + j]) & 0x7FFFFFFFu;
+              if (ka >= lo_seg) atomicSub(hist + (ka >> 19), 1u);
+            }
+          }
+        }
+      } else
       if (lv == 0 && p.use_marks) {
         // the entries of the previous support, which the walk above left out: their scores come from the override
         // list (index order), one lane per entry, straight into the segments' histograms in global memory
@@ -2015,6 +2120,157 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       }
     };
 
+    // The first digit's search, a warp per segment: the histogram is read (and cleared) from the top in runs of 512
+    // bins, 16 per lane with lane 0 at the top, down to the run that holds the segment's lower bound (nothing was
+    // counted below it).  It yields the bin b of the need-th largest entry, the entries above it and inside it, and
+    // the bin of the entry three times as far down (next round's bound).  The worker's list space is dealt out by
+    // the warp that finishes the worker's last segment, in segment order: a segment whose bin does not fit stays on
+    // the rows and takes nothing from those after it.
+    auto find_first = [&](int attempt) {
+      const int64_t nwarps = (int64_t)gridDim.x * kDenseWarps;
+      for (int64_t v = (int64_t)blockIdx.x * kDenseWarps + warp; v < nsegs; v += nwarps) {
+        const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
+        const SegState old = load_seg(a, n, s);
+        SegState* st = a.seg + (size_t)n * a.n_seg + s;
+        if (old.mode == kSegRetry) {  // the same in every lane
+          const u32 need = (u32)(a.seg_kpre[s + 1] - a.seg_kpre[s]);
+          uint4* gh = reinterpret_cast<uint4*>(a.dhist + ((size_t)n * a.n_seg + s) * kBins);
+          const int run_lo = (int)(old.lo >> 19) >> 9;
+          u32 cum = 0, b = kFull, above = 0, in_bin = 0, b_wide = kFull;
+          uint4 nx[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) nx[i] = __ldcg(gh + (kBins / 4 - 128) + (31 - lane) * 4 + i);
+          for (int run = kBins / 512 - 1; run >= run_lo; --run) {
+            uint4* g = gh + run * 128 + (31 - lane) * 4;  // this lane's 16 bins of the run
+            u32 h[16] = {nx[0].x, nx[0].y, nx[0].z, nx[0].w, nx[1].x, nx[1].y, nx[1].z, nx[1].w,
+                         nx[2].x, nx[2].y, nx[2].z, nx[2].w, nx[3].x, nx[3].y, nx[3].z, nx[3].w};
+            if (run > run_lo) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) nx[i] = __ldcg(g - 128 + i);
+            }
+            u32 sum = 0;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) sum += h[i];
+            if (sum) {  // ready for the next digit, and for the next launch
+#pragma unroll
+              for (int i = 0; i < 4; ++i) g[i] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            u32 incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+              const u32 t = __shfl_up_sync(kFull, incl, o);
+              if (lane >= o) incl += t;
+            }
+            const u32 before = cum + incl - sum;  // entries in higher bins than this lane's
+#pragma unroll
+            for (int pass = 0; pass < 2; ++pass) {
+              const bool open = pass == 0 ? b == kFull : (b_wide == kFull && need <= kFull / 3u);
+              const u32 r = pass == 0 ? need : 3u * need;
+              const u32 hit = __ballot_sync(kFull, open && before < r && r <= before + sum);
+              if (hit) {
+                const int src = __ffs(hit) - 1;
+                u32 fb = 0, fa = 0, fi = 0;
+                if (lane == src) {
+                  u32 acc = before;
+#pragma unroll
+                  for (int i = 15; i >= 0; --i) {
+                    if (acc < r && r <= acc + h[i]) { fb = (u32)(run * 512 + (31 - lane) * 16 + i); fa = acc; fi = h[i]; }
+                    acc += h[i];
+                  }
+                }
+                fb = __shfl_sync(kFull, fb, src);
+                if (pass == 0) {
+                  b = fb;
+                  above = __shfl_sync(kFull, fa, src);
+                  in_bin = __shfl_sync(kFull, fi, src);
+                } else {
+                  b_wide = fb;
+                }
+              }
+            }
+            cum += __shfl_sync(kFull, incl, 31);
+          }
+          if (lane == 0) {
+            if (b == kFull) {
+              if (old.lo == 0u) {  // fewer than k entries in the whole segment: cannot happen
+                atomicOr(&p.gctl->dense_flags, kFlagBad);
+                st->mode = kSegList; st->prefix = 0; st->need = 0; st->ties = 0;
+              } else {  // stays kSegRetry: first an octave lower, then without a bound; from the rows in any case
+                st->src = 0u;
+                st->lo = (attempt == 0 && old.lo > kOctave) ? old.lo - kOctave : 0u;
+                atomicOr(&p.gctl->dense_flags, kFlagRetry | kFlagWalk);
+              }
+            } else {
+              st->prefix = b;
+              st->need = need - above;
+              st->ties = in_bin;
+              st->mode = kSegWant;
+              // next round's lower bound: the lower edge of the bin that holds this round's 3k-th largest entry (but
+              // at least one whole bin below the threshold's own: the bins are 1/16 octave wide); if fewer than that
+              // were counted, two bins below this round's bound
+              const u32 below = b > 0u ? b - 1u : 0u;
+              u32 next;
+              if (b_wide != kFull) {  // (enough entries were counted at or above this round's bound: no need to go below it)
+                next = (b_wide < below ? b_wide : below) << 19;
+                if (LAYERED && next < old.lo) next = old.lo;
+              } else if (LAYERED) {   // a list segment whose bound lies inside the threshold's bin widens it itself
+                const u32 gap = (b << 19) > old.lo ? ((b << 19) - old.lo) >> 1 : 0u;
+                const u32 step = gap > 256u ? gap : 256u;
+                next = (b << 19) > old.lo ? (old.lo > step ? old.lo - step : 0u) : old.lo;
+              } else {
+                next = old.lo > kHintMargin ? old.lo - kHintMargin : 0u;
+              }
+              a.seg_thr[(size_t)n * a.n_seg + s] = next & ~1u;
+            }
+          }
+        }
+        // the worker's last segment to be done deals out the list space
+        u32 done = 0;
+        __syncwarp();
+        if (lane == 0) {
+          __threadfence();
+          done = atomicAdd(&p.ctl[n].seg_done, 1u);
+        }
+        done = __shfl_sync(kFull, done, 0);
+        if (done + 1u != (u32)a.n_seg) continue;
+        __threadfence();
+        u32 fill = __ldcg(&p.ctl[n].bcount);
+        for (int s0 = 0; s0 < a.n_seg; s0 += 32) {
+          const int sx = s0 + lane;
+          SegState* sp = a.seg + (size_t)n * a.n_seg + sx;
+          const bool want = sx < a.n_seg && __ldcg(&sp->mode) == kSegWant;
+          const u32 len = want ? __ldcg(&sp->ties) : 0u;
+          u32 incl = len;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const u32 t = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o) incl = (incl + t < incl) ? kFull : incl + t;  // saturating
+          }
+          const u32 all = __shfl_sync(kFull, incl, 31);
+          if (all != kFull && (u64)fill + all <= (u64)p.stride) {  // the usual case: all of them fit
+            if (want) { sp->boff = fill + incl - len; sp->mode = kSegList; }
+            fill += all;
+          } else {  // one after the other
+            for (int l = 0; l < 32; ++l) {
+              const u32 ln = __shfl_sync(kFull, len, l);
+              const bool wl = __shfl_sync(kFull, want ? 1u : 0u, l) != 0u;
+              if (!wl) continue;
+              const bool fits = (u64)fill + ln <= (u64)p.stride;
+              if (lane == l) {
+                if (fits) { sp->boff = fill; sp->mode = kSegList; }
+                else { sp->mode = kSegRows; atomicOr(&p.gctl->dense_flags, kFlagRows); }
+              }
+              if (fits) fill += ln;
+            }
+          }
+        }
+        if (lane == 0) {
+          p.ctl[n].bcount = fill;
+          p.ctl[n].seg_done = 0u;
+        }
+      }
+    };
+
     // ---- set-up: the lower bound each segment starts with ----
     for (int64_t v = (int64_t)blockIdx.x * blockDim.x + tid; v < nsegs; v += (int64_t)gridDim.x * blockDim.x) {
       const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
@@ -2032,6 +2288,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       // layer-wise: the candidate list holds every entry of the segment at or above lo, unless there was no bound to
       // gather by or the list overflowed
       st.src = (LAYERED && lo != 0u && (u64)p.ctl[n].cand_count <= (u64)p.capA) ? 1u : 0u;
+      if (LAYERED && !st.src) atomicOr(&p.gctl->dense_flags, kFlagWalk);
       st.pad[0] = st.pad[1] = st.pad[2] = 0u;
       a.seg[(size_t)n * a.n_seg + s] = st;
     }
@@ -2039,43 +2296,9 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
 
     // ---- (A) first digit; again with lo an octave lower, then with lo = 0, for the segments whose hint was too high ----
     for (int attempt = 0; attempt < 3; ++attempt) {
-      hist_pass(0, kSegRetry);
+      hist_pass(0, kSegRetry, !LAYERED || (__ldcg(&p.gctl->dense_flags) & kFlagWalk));
       grid.sync();
-      find_pass(0, kSegRetry, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin, u32 b_wide) {
-        SegState* st = a.seg + (size_t)n * a.n_seg + s;
-        if (b == kFull) {
-          if (old.lo == 0u) {  // fewer than k entries in the whole segment: cannot happen
-            atomicOr(&p.gctl->dense_flags, kFlagBad);
-            st->mode = kSegList; st->prefix = 0; st->need = 0; st->ties = 0;
-          } else {  // stays kSegRetry: first an octave lower, then without a bound; from the rows in any case
-            st->src = 0u;
-            st->lo = (attempt == 0 && old.lo > kOctave) ? old.lo - kOctave : 0u;
-            atomicOr(&p.gctl->dense_flags, kFlagRetry);
-          }
-          return;
-        }
-        st->prefix = b;
-        st->need = need - above;
-        st->ties = in_bin;
-        // next round's lower bound: the lower edge of the bin that holds this round's 3k-th largest entry; if fewer
-        // than that were counted, two bins below this round's bound
-        // (but at least one whole bin below the threshold's own: the bins are 1/16 octave wide)
-        {
-          const u32 below = b > 0u ? b - 1u : 0u;
-          const u32 edge = b_wide != kFull ? (b_wide < below ? b_wide : below) << 19
-                                           : (old.lo > kHintMargin ? old.lo - kHintMargin : 0u);
-          a.seg_thr[(size_t)n * a.n_seg + s] = edge;
-        }
-        // room for the bin's entries in the worker's B list?
-        u32 off;
-        if (reserve_list_space(&p.ctl[n].bcount, in_bin, (u64)p.stride, &off)) {
-          st->mode = kSegList;
-          st->boff = off;
-        } else {
-          st->mode = kSegRows;
-          atomicOr(&p.gctl->dense_flags, kFlagRows);
-        }
-      });
+      find_first(attempt);
       grid.sync();
       if (!(__ldcg(&p.gctl->dense_flags) & kFlagRetry)) break;  // the same in every block
       grid.sync();  // everyone has seen the flag
@@ -2083,7 +2306,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
     }
 
     // ---- (B) second pass over the rows: winners above the bin, and the bin's own entries to their list ----
-    auto compact_pass = [&](u32 want_mode) {
+    auto compact_pass = [&](u32 want_mode, bool walk) {
       int cur_n = -1, cur_s = -1;
       // During the walk a thread that holds an entry at or above the bin's lower edge puts it into its warp's
       // staging list itself (one shared-memory counter).  When the list is half full, or the segment changes, the
@@ -2142,7 +2365,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       __syncwarp();
       SegState st;
       st.mode = ~0u;
-      for (int64_t w = w_begin; w < w_end; ++w) {
+      for (int64_t w = walk ? w_begin : w_end; w < w_end; ++w) {
         const DenseTile t = dense_tile(a, s_flagged, w);
         if (t.n != cur_n || t.s != cur_s) {
           if (cur_n >= 0 && st.mode == want_mode) flush(cur_n, cur_s, st);
@@ -2168,53 +2391,123 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       }
       if (cur_n >= 0 && st.mode == want_mode) flush(cur_n, cur_s, st);
       u32 cntA = 0;  // from here on the lists are filled by ballot: warp-uniform fill
+      if (LAYERED && want_mode == kSegList) {
+        // Layer-wise mode: the candidate lists of the segments fed from them, then the override list, as runs of
+        // 32-entry tasks over all flagged workers, dealt to the warps of the grid in contiguous pieces (as in the
+        // histogram pass).  Each warp keeps the first half of its staging space for the winners it finds; the
+        // other halves hold, when they fit, what is needed of every segment's state.
+        __syncthreads();  // every warp has written out what the walk above staged
+        u64* listL = s_stage + (size_t)warp * kWarpList;
+        uint4* t_seg = reinterpret_cast<uint4*>(s_stage + (size_t)kDenseWarps * kWarpList);  // [nsegs]: prefix | flags, bound, list offset, list length
+        u32* t_end = s_hist;                                                                // [n_seg]
+        const bool fast = (u64)nsegs * 2u <= (u64)kDenseWarps * kWarpList && a.n_seg <= kBins;
+        constexpr u32 kPart = 1u << 31, kFed = 1u << 30;
+        auto pack = [&](const SegState& sg) {
+          return make_uint4(sg.prefix | (sg.mode == kSegList ? kPart : 0u) | (sg.src ? kFed : 0u), sg.lo, sg.boff, sg.ties);
+        };
+        if (fast) {
+          for (int i = tid; i < a.n_seg; i += blockDim.x) t_end[i] = (u32)a.seg_end[i];
+          for (int64_t v = tid; v < nsegs; v += blockDim.x)
+            t_seg[v] = pack(load_seg(a, (int)s_flagged[v / a.n_seg], (int)(v % a.n_seg)));
+          __syncthreads();
+        }
+        auto seg_of = [&](u32 j) -> int {
+          if (!fast) return dense_seg_of_index(a.seg_end, a.n_seg, (int64_t)j);
+          int lo = 0, hi = a.n_seg - 1;  // the first segment whose end lies beyond j
+          while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (t_end[mid] <= j) lo = mid + 1; else hi = mid;
+          }
+          return lo;
+        };
+        auto info_of = [&](int64_t f, int n, int s) -> uint4 {
+          return fast ? t_seg[f * a.n_seg + s] : pack(load_seg(a, n, s));
+        };
+        int cur = -1;  // the worker whose winners the warp is staging
+        auto flush_L = [&]() {
+          if (cur >= 0) stage_flush(listL, cntA, &p.ctl[cur].acount, p.ovr_comp + (size_t)cur * p.k, (u64)k, lane);
+        };
+        // one task's entries (c: composite, live: this lane has one; fed_only: candidates count for list-fed segments only)
+        auto place_task = [&](int64_t f, int n, u64 c, bool live, bool fed_only) {
+          if (n != cur) { flush_L(); cur = n; }
+          const u32 key = (u32)(c >> 32), j = composite_idx(c);
+          const int s = (live && a.n_seg > 1) ? seg_of(j) : 0;
+          uint4 sg = make_uint4(0u, 0u, 0u, 0u);
+          if (live) sg = info_of(f, n, s);
+          const bool part = (sg.x & kPart) && (!fed_only || (sg.x & kFed));
+          const u32 prefix = sg.x & 0x00FFFFFFu;
+          const bool win = part && (key >> 19) > prefix;
+          const bool bin = part && (key >> 19) == prefix && key >= sg.y;
+          if (win) set_winner(p.mask_new + (size_t)n * p.W, j, p.d);
+          const u32 act = __ballot_sync(kFull, bin);
+          if (bin) {  // the bin's entries to their segment's list: lanes of one segment reserve their places together
+            const u32 peers = __match_any_sync(act, (u32)s);
+            const int leader = __ffs(peers) - 1;
+            u32 base = 0;
+            if (lane == leader) base = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, (u32)__popc(peers));
+            base = __shfl_sync(peers, base, leader);
+            const u32 pos = base + (u32)__popc(peers & ((1u << lane) - 1u));
+            if (RT_INB(pos < sg.w)) p.candB[(size_t)n * p.stride + sg.z + pos] = c;
+          }
+          if (__any_sync(kFull, win)) {
+            stage_add(listL, cntA, win, c, lane);
+            if (cntA >= (u32)(kWarpList - 32)) flush_L();
+          }
+        };
+        const int64_t gw = (int64_t)blockIdx.x * kDenseWarps + warp, nwarps = (int64_t)gridDim.x * kDenseWarps;
+        {  // candidates
+          const int64_t tasks = s_cbase[nf];
+          const int64_t per = (tasks + nwarps - 1) / nwarps;
+          const int64_t t0 = gw * per, t1 = t0 + per < tasks ? t0 + per : tasks;
+          int64_t f = 0;
+          if (t0 < t1) {
+            int64_t lo = 0, hi = nf;  // the worker whose tasks include t0
+            while (hi - lo > 1) {
+              const int64_t mid = (lo + hi) >> 1;
+              if ((int64_t)s_cbase[mid] <= t0) lo = mid; else hi = mid;
+            }
+            f = lo;
+          }
+          auto fetch = [&](int64_t t, int64_t& ff, bool& live) -> u64 {
+            live = false;
+            if (t >= t1) return 0ull;
+            while (t >= (int64_t)s_cbase[ff + 1]) ++ff;
+            const int n = (int)s_flagged[ff];
+            const int64_t i = (t - (int64_t)s_cbase[ff]) * 32 + lane;
+            live = i < (int64_t)p.ctl[n].cand_count;
+            return live ? __ldcg(p.candA + (size_t)n * p.stride + i) : 0ull;
+          };
+          int64_t f_next = f;
+          bool live_next = false;
+          u64 c_next = fetch(t0, f_next, live_next);
+          for (int64_t t = t0; t < t1; ++t) {
+            const u64 c = c_next;
+            const bool live = live_next;
+            f = f_next;
+            c_next = fetch(t + 1, f_next, live_next);
+            place_task(f, (int)s_flagged[f], c, live, true);
+          }
+        }
+        if (p.use_marks) {  // the previous support: scores from the override list
+          const int64_t per_w = (p.k + 31) / 32, tasks = nf * per_w;
+          const int64_t per = (tasks + nwarps - 1) / nwarps;
+          const int64_t t0 = gw * per, t1 = t0 + per < tasks ? t0 + per : tasks;
+          for (int64_t t = t0; t < t1; ++t) {
+            const int64_t f = t / per_w;
+            const int n = (int)s_flagged[f];
+            const int64_t i = (t - f * per_w) * 32 + lane;
+            const bool live = i < p.k;
+            const int32_t j = live ? p.prev_idx[(size_t)n * p.k + i] : 0;
+            const u32 key = live ? __ldcg(&p.ovr_key[(size_t)n * p.k + i]) : 0u;
+            place_task(f, n, make_composite(key, (u32)j), live, false);
+          }
+        }
+        flush_L();
+        return;
+      }
       auto flush_A2 = [&](int n) {
         stage_flush(listA, cntA, &p.ctl[n].acount, p.ovr_comp + (size_t)n * p.k, (u64)k, lane);
       };
-      if (LAYERED && want_mode == kSegList) {  // the segments fed from the candidate list
-        for (int64_t f = 0; f < nf; ++f) {
-          const int n = (int)s_flagged[f];
-          const u32 cc = p.ctl[n].cand_count;
-          if ((u64)cc > (u64)p.capA) continue;
-          const u64* cand = p.candA + (size_t)n * p.stride;
-          u32* mask = p.mask_new + (size_t)n * p.W;
-          for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + (tid & ~31); i0 < (int64_t)cc; i0 += (int64_t)gridDim.x * blockDim.x) {
-            const int64_t i = i0 + lane;
-            const bool live = i < (int64_t)cc;
-            const u64 c = live ? __ldcg(&cand[i]) : 0ull;
-            const u32 key = (u32)(c >> 32), j = composite_idx(c);
-            const int s = (live && a.n_seg > 1) ? dense_seg_of_index(a.seg_end, a.n_seg, (int64_t)j) : 0;
-            bool win = false, bin = false;
-            SegState st;
-            st.boff = 0; st.ties = 0;
-            if (live) {
-              st = load_seg(a, n, s);
-              if (st.mode == kSegList && st.src) {
-                win = (key >> st.sh) > st.prefix;
-                bin = (key >> st.sh) == st.prefix && key >= st.lo;
-              }
-            }
-            if (win) set_winner(mask, j, p.d);
-            {  // the bin's entries to their segment's list: lanes of one segment reserve their places together
-              const u32 act = __ballot_sync(kFull, bin);
-              if (bin) {
-                const u32 peers = __match_any_sync(act, (u32)s);
-                const int leader = __ffs(peers) - 1;
-                u32 base = 0;
-                if (lane == leader) base = atomicAdd(&a.seg[(size_t)n * a.n_seg + s].bfill, (u32)__popc(peers));
-                base = __shfl_sync(peers, base, leader);
-                const u32 pos = base + (u32)__popc(peers & ((1u << lane) - 1u));
-                if (RT_INB(pos < st.ties)) p.candB[(size_t)n * p.stride + st.boff + pos] = c;
-              }
-            }
-            if (__any_sync(kFull, win)) {
-              stage_add(listA, cntA, win, c, lane);
-              if (cntA >= (u32)(kWarpList - 32)) flush_A2(n);
-            }
-          }
-          flush_A2(n);
-        }
-      }
       if (p.use_marks) {  // the same for the entries of the previous support, from the override list
         for (int64_t f = 0; f < nf; ++f) {
           const int n = (int)s_flagged[f];
@@ -2260,12 +2553,35 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         }
       }
     };
-    compact_pass(kSegList);
     const u32 flags0 = __ldcg(&p.gctl->dense_flags);  // written before the last barrier
-    if (flags0 & kFlagRows) hist_pass(1, kSegRows);
+    compact_pass(kSegList, !LAYERED || (flags0 & kFlagWalk));
+    if (flags0 & kFlagRows) hist_pass(1, kSegRows, true);
     grid.sync();
 
     // ---- (C) per list segment: the `need` largest composites of its in-bin list win ----
+    // Layer-wise mode: the lower bound a list segment leaves for the next round.  Error feedback packs more and more
+    // entries right under the threshold, so the bound goes by rank, not by magnitude: it is the key of the entry
+    // max(2 k_s, 32) places below the threshold in the segment's in-bin list (bound_rank: its place in that list).
+    // A list too short for that (few entries at or above this round's bound) widens the gap between the bound and
+    // the threshold key by a half, as long as the bound lies inside the threshold's bin; otherwise the bin edge that
+    // the first digit's search left stands.
+    auto bound_rank = [&](const SegState& sg, int s) -> u32 {
+      const u32 ks = (u32)(a.seg_kpre[s + 1] - a.seg_kpre[s]);
+      const u32 more = ks > 16u ? (ks > kFull / 4u ? kFull / 2u : 2u * ks) : 32u;
+      return sg.need + more < more ? kFull : sg.need + more;
+    };
+    auto leave_rank_bound = [&](int n, int s, const SegState& sg, u32 key_r) {  // one thread
+      if (!LAYERED || sg.mode != kSegList) return;
+      a.seg_thr[(size_t)n * a.n_seg + s] = key_r & ~1u;
+    };
+    auto leave_wider_bound = [&](int n, int s, const SegState& sg, u32 t_key) {  // one thread
+      if (!LAYERED || sg.mode != kSegList) return;
+      const u32 edge = sg.prefix << 19;
+      if (sg.lo <= edge) return;
+      const u32 gap = t_key > sg.lo ? (t_key - sg.lo) >> 1 : 0u;
+      const u32 step = gap > 256u ? gap : 256u;
+      a.seg_thr[(size_t)n * a.n_seg + s] = (sg.lo - edge > step ? sg.lo - step : edge) & ~1u;
+    };
     auto list_select = [&](u32 want_mode) {
      for (int64_t v = blockIdx.x; v < nsegs; v += gridDim.x) {
       const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
@@ -2278,6 +2594,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         if (tid == 0) atomicOr(&p.gctl->dense_flags, kFlagBad);
         continue;
       }
+      const u32 r_bound = LAYERED ? bound_rank(st, s) : kFull;  // place in the list of the entry whose key is the next bound
       if (count <= blockDim.x) {
         // a short list (the usual case): every thread ranks its entry against all others in shared memory; the
         // entry with `above` larger ones before it takes place `above` among the segment's winners from this list
@@ -2290,6 +2607,10 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         if ((u32)tid < count) {
           u32 above = 0;
           for (u32 j = 0; j < count; ++j) above += items[j] > mine ? 1u : 0u;
+          if (count >= r_bound ? above + 1u == r_bound : above + 1u == st.need) {
+            if (count >= r_bound) leave_rank_bound(n, s, st, (u32)(mine >> 32));
+            else leave_wider_bound(n, s, st, (u32)(mine >> 32));
+          }
           if (above < st.need) {
             set_winner(mask, composite_idx(mine), p.d);
             if (RT_INB((u64)s_cnt + above < (u64)k)) p.ovr_comp[(size_t)n * p.k + s_cnt + above] = mine;
@@ -2298,50 +2619,140 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         __syncthreads();
         continue;
       }
-      // the need-th largest composite, byte by byte (the list stays where it is)
+      // A longer list: the need-th largest composite T, digit by digit: the key bits below the digits already fixed
+      // first (19 as 11 + 8, or 7), then, only while entries of one key are still to be told apart, the index
+      // bytes.  A digit whose bin is taken whole ends the search: the bin's lower edge is T.  The entries that are
+      // still in play sit in shared memory (the warps' staging space, free in this phase): the whole list if it
+      // fits, otherwise what the first digits leave of it, gathered in the pass that also emits the entries above.
+      u64* items = s_stage;
+      constexpr u32 kItems = (u32)(kDenseWarps * 2 * kWarpList);
+      u64* A = p.ovr_comp + (size_t)n * p.k;
+      __syncthreads();
+      if (tid == 0) {
+        s_res[0] = atomicAdd(&p.ctl[n].acount, st.need);  // the segment's places in the worker's winner list
+        s_cnt = 0;                                        // winners placed so far
+        s_nf2 = 0;                                        // entries gathered in shared memory
+      }
+      __syncthreads();
+      const u32 abase = s_res[0];
+      auto emit = [&](bool won, u64 c) {  // every lane of the warp
+        const u32 mw = __ballot_sync(kFull, won);
+        if (!mw) return;
+        u32 at = 0;
+        if (lane == 0) at = atomicAdd(&s_cnt, (u32)__popc(mw));
+        at = __shfl_sync(kFull, at, 0) + (u32)__popc(mw & ((1u << lane) - 1u));
+        if (won) {
+          set_winner(mask, composite_idx(c), p.d);
+          if (RT_INB(at < st.need && (u64)abase + at < (u64)k)) A[(u64)abase + at] = c;
+        }
+      };
+      const u32 rounded = (count + 31u) & ~31u;
+      if (st.need >= count) {  // all of them
+        for (u32 i = tid; i < rounded; i += blockDim.x) emit(i < count, i < count ? __ldcg(&list[i]) : 0ull);
+        __syncthreads();
+        continue;
+      }
+      bool in_smem = count <= kItems;
+      u32 m = count;  // entries in play
+      if (in_smem) {
+        for (u32 i0 = tid; i0 < count; i0 += 4u * blockDim.x) {  // four loads in flight
+          u64 v[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) v[q] = i0 + q * blockDim.x < count ? __ldcg(&list[i0 + q * blockDim.x]) : 0ull;
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (i0 + q * blockDim.x < count) items[i0 + q * blockDim.x] = v[q];
+        }
+      }
       u32 need = st.need;
-      u64 prefix = 0ull;
-      bool bad = false;
-      if (need < count) {
-        for (int shift = 56; shift >= 0 && !bad; shift -= 8) {
+      u64 prefix = (u64)st.prefix;  // every entry of the list has these digits
+      int top = 32 + (int)st.sh;    // composite bits below the prefix
+      bool bad = false, have_T = false;
+      while (top > 0) {
+        const int width = top > 32 ? (top - 32 > 11 ? 11 : top - 32) : 8;
+        const int shift = top - width, bins = 1 << width;
+        __syncthreads();
+        for (int i = tid; i < bins; i += blockDim.x) s_hist[i] = 0;
+        __syncthreads();
+        for (u32 i = tid; i < m; i += blockDim.x) {
+          const u64 c = in_smem ? items[i] : __ldcg(&list[i]);
+          if ((c >> top) == prefix) atomicAdd(&s_hist[(u32)(c >> shift) & (u32)(bins - 1)], 1u);
+        }
+        __syncthreads();
+        block_find_from_top(s_hist, bins, need, s_scan, s_res + 1);
+        const u32 bb = s_res[1], above = s_res[2];
+        if (bb == kFull) { bad = true; break; }  // the same in every thread
+        if (LAYERED && top == 32 + (int)st.sh && count >= r_bound && shift >= 32) {
+          // (first digit: the histogram covers the whole list) the sub-bin of the entry that gives the next bound
+          __syncthreads();  // everyone has read the first search's result
+          block_find_from_top(s_hist, bins, r_bound, s_scan, s_res + 1);
+          if (tid == 0 && s_res[1] != kFull)
+            leave_rank_bound(n, s, st, (u32)((((prefix << width) | (u64)s_res[1]) << (shift - 32))));
           __syncthreads();
-          for (int i = tid; i < 256; i += blockDim.x) s_hist[i] = 0;
+        }
+        need -= above;
+        prefix = (prefix << width) | (u64)bb;
+        top = shift;
+        const u32 in_bin = s_hist[bb];
+        if (in_bin == need) break;  // all of this bin win
+        if (in_bin <= blockDim.x) {
+          // few entries are left in play: they are ranked against one another, and the need-th largest is T
+          u64* ties = reinterpret_cast<u64*>(s_hist);
+          __syncthreads();  // everyone has read the histogram
+          if (tid == 0) s_nf2 = 0;
           __syncthreads();
-          for (u32 i = tid; i < count; i += blockDim.x) {
-            const u64 c = __ldcg(&list[i]);
-            if (shift == 56 || (c >> (shift + 8)) == prefix) atomicAdd(&s_hist[(u32)(c >> shift) & 255u], 1u);
+          for (u32 i = tid; i < m; i += blockDim.x) {
+            const u64 c = in_smem ? items[i] : __ldcg(&list[i]);
+            if ((c >> top) == prefix) {
+              const u32 at = atomicAdd(&s_nf2, 1u);
+              if (RT_INB(at < blockDim.x)) ties[at] = c;
+            }
           }
           __syncthreads();
-          block_find_from_top(s_hist, 256, need, s_scan, s_res);
-          const u32 b = s_res[0], above = s_res[1];
-          if (b == kFull) { bad = true; break; }  // the same in every thread
-          need -= above;
-          prefix = (prefix << 8) | (u64)b;
+          if (s_nf2 != in_bin) { bad = true; break; }  // the same in every thread
+          if ((u32)tid < in_bin) {
+            const u64 mine = ties[tid];
+            u32 above = 0;
+            for (u32 j = 0; j < in_bin; ++j) above += ties[j] > mine ? 1u : 0u;
+            if (above + 1u == need) s_T = mine;
+          }
+          __syncthreads();
+          have_T = true;
+          break;
+        }
+        if (!in_smem && in_bin <= kItems) {
+          // one pass over the list: what lies above the digits found so far wins now, what matches them moves to
+          // shared memory and the search goes on there
+          for (u32 i = tid; i < rounded; i += blockDim.x) {
+            const u64 c = i < count ? __ldcg(&list[i]) : 0ull;
+            const u64 hi = c >> top;
+            emit(i < count && hi > prefix, c);
+            const u32 mk = __ballot_sync(kFull, i < count && hi == prefix);
+            if (mk) {
+              u32 at = 0;
+              if (lane == 0) at = atomicAdd(&s_nf2, (u32)__popc(mk));
+              at = __shfl_sync(kFull, at, 0) + (u32)__popc(mk & ((1u << lane) - 1u));
+              if (i < count && hi == prefix && RT_INB(at < kItems)) items[at] = c;
+            }
+          }
+          in_smem = true;
+          m = in_bin;
         }
       }
       if (bad) {
         if (tid == 0) atomicOr(&p.gctl->dense_flags, kFlagBad);
         continue;
       }
-      // winners: at or above that composite (every entry if all are needed); they join the worker's winner list
       __syncthreads();
-      if (tid == 0) s_cnt = atomicAdd(&p.ctl[n].acount, st.need);
-      __syncthreads();
-      const u32 abase = s_cnt;
-      u64* A = p.ovr_comp + (size_t)n * p.k;
-      u32 carry = 0;
-      for (u32 i0 = 0; i0 < count; i0 += blockDim.x) {
-        const u32 i = i0 + tid;
-        const u64 c = i < count ? __ldcg(&list[i]) : 0ull;
-        const bool won = i < count && c >= prefix;
-        u32 total;
-        const u32 at = block_excl_scan(won ? 1u : 0u, s_scan, &total);
-        if (won) {
-          set_winner(mask, composite_idx(c), p.d);
-          if (RT_INB((u64)abase + carry + at < (u64)k)) A[(u64)abase + carry + at] = c;
-        }
-        carry += total;
+      const u64 T = have_T ? s_T : prefix << top;  // the lowest composite that wins
+      if (tid == 0 && count < r_bound) leave_wider_bound(n, s, st, (u32)(T >> 32));
+      const u32 mr = (m + 31u) & ~31u;
+      for (u32 i = tid; i < mr; i += blockDim.x) {
+        const u64 c = i < m ? (in_smem ? items[i] : __ldcg(&list[i])) : 0ull;
+        emit(i < m && c >= T, c);
       }
+      __syncthreads();
+      if (tid == 0 && s_cnt != st.need) atomicOr(&p.gctl->dense_flags, kFlagBad);
      }
     };
     list_select(kSegList);
@@ -2367,8 +2778,8 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       });
       grid.sync();
       const u32 flags_b = __ldcg(&p.gctl->dense_flags);
-      compact_pass(kSegList2);
-      if (flags_b & kFlagRows2) hist_pass(2, kSegRows);
+      compact_pass(kSegList2, true);
+      if (flags_b & kFlagRows2) hist_pass(2, kSegRows, true);
       grid.sync();
       list_select(kSegList2);
      if (flags_b & kFlagRows2) {
@@ -2505,7 +2916,11 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         post_prefix_segment(p, (int)s_flagged[it / a.emit_segments], (u32)(it % a.emit_segments), seg_units, lane);
       grid.sync();
       u32* s_segbase = s_hist;
-      for (int64_t f = 0; f < nf; ++f) {
+      // a team of blocks per worker (all workers at once while there are at most as many as blocks)
+      const int64_t teams = nf < (int64_t)gridDim.x ? (int64_t)gridDim.x / nf : 1;
+      const int64_t slots = (int64_t)gridDim.x / teams;
+      const u32 member = (u32)(blockIdx.x % teams);
+      for (int64_t f = blockIdx.x / teams; f < nf; f += slots) {  // the same in every thread of the block
         const int n = (int)s_flagged[f];
         constexpr int kSegPer = kMaxSegments / kDenseThreads;  // consecutive mask segments per thread
         u32 mine[kSegPer], sum = 0, total;
@@ -2522,16 +2937,15 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
           const u32 sg = (u32)(kSegPer * tid + i);
           if (sg < a.emit_segments) {
             s_segbase[sg] = base;
-            if (blockIdx.x == 0) p.segbase[(size_t)n * kMaxSegments + sg] = base;  // for k_aggregate
+            if (member == 0u) p.segbase[(size_t)n * kMaxSegments + sg] = base;  // for k_aggregate
           }
           base += mine[i];
         }
         __syncthreads();
         if (total != k) {
-          if (blockIdx.x == 0 && tid == 0) atomicOr(&p.gctl->err, kErrCountMismatch);
+          if (member == 0u && tid == 0) atomicOr(&p.gctl->err, kErrCountMismatch);
         } else {
-          post_emit(p, n, blockIdx.x * blockDim.x + tid, gridDim.x * blockDim.x, 0u, 0u, true, 0u, 0u, 0u, s_segbase,
-                    seg_units);
+          post_emit(p, n, member * blockDim.x + tid, (u32)teams * blockDim.x, 0u, 0u, true, 0u, 0u, 0u, s_segbase, seg_units);
         }
         __syncthreads();
       }
@@ -3259,7 +3673,7 @@ int step_impl(regtopk_ctx* c, const void* grads, int64_t grad_ld, int32_t* out_i
     // worker asked for the dense path.
     DenseArgs da;
     da.p = pa; da.N = c->N; da.n_seg = (int)L.n_seg; da.finish = pa.wide ? 0 : 1;
-    da.emit_segments = (u32)(c->cluster * (kBlockPost / 32));
+    da.emit_segments = c->layered ? (u32)kMaxSegments : (u32)(c->cluster * (kBlockPost / 32));
     da.tiles = L.tiles;
     da.seg_end = at<int64_t>(c, L.off_seg_end); da.seg_kpre = at<int64_t>(c, L.off_seg_kpre);
     da.seg_tile0 = at<int64_t>(c, L.off_seg_tile0);
@@ -3338,8 +3752,9 @@ int regtopk_aggregate_update(regtopk_ctx* c, float* theta, float eta, float* out
   a.cur_idx = at<int32_t>(c, L.off_idx[c->cur]); a.cur_val = at<float>(c, L.off_val[c->cur]);
   a.prev_idx = at<int32_t>(c, L.off_idx[c->cur ^ 1]);
   a.bitmask = at<u32>(c, L.off_mask[c->cur]); a.qprefix = at<u32>(c, L.off_qprefix); a.segbase = at<u32>(c, L.off_segbase);
-  {  // segments of the mask row as the emission cut them: one per warp of the k_post cluster, kMaxSegments in wide mode
-    const int64_t nseg = c->many_pairs ? kMaxSegments : (int64_t)c->cluster * (kBlockPost / 32);
+  {  // segments of the mask row as the emission cut them: one per warp of the k_post cluster; kMaxSegments in wide
+     // mode and in layer-wise mode, where the whole grid emits
+    const int64_t nseg = (c->many_pairs || c->layered) ? kMaxSegments : (int64_t)c->cluster * (kBlockPost / 32);
     a.seg_units = ((L.W >> 3) + nseg - 1) / nseg;
   }
   a.W = L.W;
