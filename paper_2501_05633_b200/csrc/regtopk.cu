@@ -2674,9 +2674,21 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         __syncthreads();
         for (int i = tid; i < bins; i += blockDim.x) s_hist[i] = 0;
         __syncthreads();
-        for (u32 i = tid; i < m; i += blockDim.x) {
-          const u64 c = in_smem ? items[i] : __ldcg(&list[i]);
-          if ((c >> top) == prefix) atomicAdd(&s_hist[(u32)(c >> shift) & (u32)(bins - 1)], 1u);
+        if (in_smem) {
+          for (u32 i = tid; i < m; i += blockDim.x) {
+            const u64 c = items[i];
+            if ((c >> top) == prefix) atomicAdd(&s_hist[(u32)(c >> shift) & (u32)(bins - 1)], 1u);
+          }
+        } else {
+          for (u32 i0 = tid; i0 < m; i0 += 4u * blockDim.x) {  // four loads in flight
+            u64 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[q] = i0 + q * blockDim.x < m ? __ldcg(&list[i0 + q * blockDim.x]) : 0ull;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              if (i0 + q * blockDim.x < m && (v[q] >> top) == prefix)
+                atomicAdd(&s_hist[(u32)(v[q] >> shift) & (u32)(bins - 1)], 1u);
+          }
         }
         __syncthreads();
         block_find_from_top(s_hist, bins, need, s_scan, s_res + 1);
@@ -2723,16 +2735,24 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         if (!in_smem && in_bin <= kItems) {
           // one pass over the list: what lies above the digits found so far wins now, what matches them moves to
           // shared memory and the search goes on there
-          for (u32 i = tid; i < rounded; i += blockDim.x) {
-            const u64 c = i < count ? __ldcg(&list[i]) : 0ull;
-            const u64 hi = c >> top;
-            emit(i < count && hi > prefix, c);
-            const u32 mk = __ballot_sync(kFull, i < count && hi == prefix);
-            if (mk) {
-              u32 at = 0;
-              if (lane == 0) at = atomicAdd(&s_nf2, (u32)__popc(mk));
-              at = __shfl_sync(kFull, at, 0) + (u32)__popc(mk & ((1u << lane) - 1u));
-              if (i < count && hi == prefix && RT_INB(at < kItems)) items[at] = c;
+          for (u32 i0 = tid; i0 < rounded; i0 += 4u * blockDim.x) {  // four loads in flight; whole warps take each step
+            u64 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[q] = i0 + q * blockDim.x < count ? __ldcg(&list[i0 + q * blockDim.x]) : 0ull;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const u32 i = i0 + q * blockDim.x;
+              if (i - lane >= rounded) break;  // the same in every lane
+              const u64 c = v[q];
+              const u64 hi = c >> top;
+              emit(i < count && hi > prefix, c);
+              const u32 mk = __ballot_sync(kFull, i < count && hi == prefix);
+              if (mk) {
+                u32 at = 0;
+                if (lane == 0) at = atomicAdd(&s_nf2, (u32)__popc(mk));
+                at = __shfl_sync(kFull, at, 0) + (u32)__popc(mk & ((1u << lane) - 1u));
+                if (i < count && hi == prefix && RT_INB(at < kItems)) items[at] = c;
+              }
             }
           }
           in_smem = true;
