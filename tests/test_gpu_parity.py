@@ -334,6 +334,42 @@ def test_layerwise_scaled_workloads(name):
     run_parity((s.next() for _ in range(6)), w.d, w.N, 0, w.mu, layers=L)
 
 
+def _drift_rounds(N, d, T, seed, scales):
+    """A fixed direction plus noise, as error feedback meets it in training: unsent entries pile up under the
+    thresholds round after round.  scales[t] multiplies round t (a missing entry is 1)."""
+    g = torch.Generator().manual_seed(seed)
+    base = torch.randn(d, generator=g)
+    for t in range(T):
+        v = 0.5 * base + torch.randn((N, d), generator=g)
+        yield (v * float(scales.get(t, 1.0))).contiguous()
+
+
+def test_layerwise_long_in_bin_lists_over_many_rounds():
+    """A layer with k_l = 30,000: its in-bin list is ranked from shared memory (more than a block's worth of entries)
+    and, when it outgrows that, gathered after a first digit; the bounds for the next round go by rank."""
+    sizes = [1_500_000, 300, 64, 200_000, 17]
+    d = int(sum(sizes))
+    run_parity(_drift_rounds(2, d, 10, seed=31, scales={}), d, 2, 0, 4.0, layers=_layers_of(sizes, 0.02), threads=8)
+
+
+def test_layerwise_thresholds_that_fall_and_lists_that_overflow():
+    """Rounds whose gradients shrink a thousandfold with the sign turned (the accumulators and with them the layers'
+    thresholds fall under the bounds left for the streaming pass: those layers are counted again from the rows) and
+    rounds that grow a hundredfold (every entry passes the old bounds and the candidate lists overflow)."""
+    sizes = [120_000, 64, 64, 260_000, 1000, 30_011]
+    d = int(sum(sizes))
+    scales = {3: -1e-3, 4: -1e-3, 6: 100.0, 8: 1e-2, 9: -30.0}
+    run_parity(_drift_rounds(3, d, 11, seed=5, scales=scales), d, 3, 0, 4.0, layers=_layers_of(sizes, 0.01), threads=8)
+
+
+@pytest.mark.parametrize("N,n_layers", [(24, 100), (40, 450)])
+def test_layerwise_more_segments_than_the_shared_tables_hold(N, n_layers):
+    rng = np.random.default_rng(N)
+    sizes = [int(x) for x in rng.integers(20, 90, size=n_layers)]
+    d = int(sum(sizes))
+    run_parity(_drift_rounds(N, d, 5, seed=N, scales={}), d, N, 0, 4.0, layers=_layers_of(sizes, 0.1), threads=8)
+
+
 def test_layerwise_argument_errors():
     for layers in [([10, 5], [1, 1]), ([5, 9], [1, 1]), ([5, 10], [0, 1]), ([5, 10], [6, 1]), ([5, 5, 10], [1, 1, 1])]:
         with pytest.raises(RegTopKError):
