@@ -370,6 +370,15 @@ def test_layerwise_more_segments_than_the_shared_tables_hold(N, n_layers):
     run_parity(_drift_rounds(N, d, 5, seed=N, scales={}), d, N, 0, 4.0, layers=_layers_of(sizes, 0.1), threads=8)
 
 
+def test_layerwise_sixty_rounds_on_a_tensor_table():
+    """Long enough for the bounds that each layer's selection leaves for the next round to settle and to be missed now
+    and then (ResNet-18's tensor table scaled down, error feedback ageing over 60 rounds)."""
+    w = synth.workload("resnet18", scale_to=400_000)
+    L = _layers_of(w.shapes, 0.01)
+    s = synth.GradientStream(w, device="cpu", seed=23, pad_to=8)
+    run_parity((s.next() for _ in range(60)), w.d, w.N, 0, w.mu, layers=L, threads=8)
+
+
 def test_layerwise_argument_errors():
     for layers in [([10, 5], [1, 1]), ([5, 9], [1, 1]), ([5, 10], [0, 1]), ([5, 10], [6, 1]), ([5, 5, 10], [1, 1, 1])]:
         with pytest.raises(RegTopKError):
