@@ -803,3 +803,63 @@ def test_full_size_certified(name, ki, rounds):
             eps_before = lib.residual().cpu().numpy()
         del grads
     assert lib.stats()["dense_select_workers"] == 0
+
+
+# ---- layer-wise selection at the benchmark's sizes ----------------------------------------------------------------
+def test_full_size_layerwise_resnet18():
+    """Every tensor of the ResNet-18 table a layer with 0.1 % of its size, as `bench.py --select layerwise` runs it:
+    round 0 from the rows, the later rounds from the candidate lists."""
+    w = synth.workload("resnet18")
+    L = _layers_of(w.shapes, w.sparsity[0])
+    s = synth.GradientStream(w, device="cuda", seed=0, pad_to=32)
+    run_parity((s.next() for _ in range(10)), w.d, w.N, 0, w.mu, layers=L, threads=8)
+
+
+def test_full_size_layerwise_certified_gpt2():
+    """The GPT-2 table (bf16 gradients, 148 layers with 0.01 % each) at full size, certified layer by layer without a
+    sort: inside every layer no entry outside the library's selection ranks before its last-ranked entry."""
+    import psutil
+    from oracle.oracle import default as oracle_default
+    w = synth.workload("gpt2")
+    if psutil.virtual_memory().available < 5 * w.N * w.d * 4:
+        pytest.skip("not enough host memory for the element-wise checks")
+    ends, ks = _layers_of(w.shapes, w.sparsity[0])
+    k = int(sum(ks))
+    api = oracle_default()
+    s = synth.GradientStream(w, device="cuda", seed=0, pad_to=32)
+    lib = RegTopK(w.d, w.N, 0, mu=w.mu, grad_dtype=torch.bfloat16, layers=(ends, ks))
+    omega = np.full(w.N, np.float32(1.0) / np.float32(w.N), np.float32)
+    eps_before = np.zeros((w.N, w.d), np.float32)
+    prev, g_prev = None, None
+    for t in range(3):
+        grads = s.next()
+        idx, val = lib.worker_step(grads)
+        lib.status()
+        idx_h, val_h = idx.cpu().numpy(), val.cpu().numpy()
+        eps_after = lib.residual()
+        for n in range(w.N):
+            g_view = grads[n, : w.d].cpu().view(torch.int16).numpy().view(np.uint16)
+            pi, pv = (None, None) if prev is None else (prev[0][n], prev[1][n])
+            a, sc = api.scores(g_view, eps_before[n], pi, pv, g_prev, w.mu, float(omega[n]))
+            assert np.all(np.diff(idx_h[n]) > 0), f"worker {n}: indices not ascending"
+            cut = np.searchsorted(idx_h[n], np.asarray([0] + ends))
+            begin = 0
+            for l, end in enumerate(ends):
+                sel = idx_h[n][cut[l]: cut[l + 1]] - begin
+                assert sel.shape[0] == ks[l], f"worker {n} layer {l}: {sel.shape[0]} selected, {ks[l]} wanted"
+                assert api.mask_certificate(sc[begin:end], sel) == ks[l], f"worker {n} layer {l}: not its k largest scores"
+                begin = end
+            assert np.array_equal(val_h[n].view(np.uint32), a[idx_h[n]].view(np.uint32)), f"worker {n}: sent values"
+            a[idx_h[n]] = 0.0
+            assert np.array_equal(eps_after[n].cpu().numpy().view(np.uint32), a.view(np.uint32)), f"worker {n}: residual"
+            del a, sc
+        agg = lib.aggregate().cpu().numpy()
+        want = api.aggregate(w.d, omega, idx_h, val_h)
+        assert np.array_equal(agg.view(np.uint32), want.view(np.uint32)), "aggregate"
+        lib.status()
+        prev, g_prev = (idx_h, val_h), agg
+        if t < 2:
+            eps_before = lib.residual().cpu().numpy()
+        del grads
+    assert k == lib.k
+    lib.close()
