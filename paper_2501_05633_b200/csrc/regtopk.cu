@@ -1567,14 +1567,17 @@ __global__ void __launch_bounds__(256) k_unzip(UnzipArgs p) {
 //
 // Per segment:
 //   (A) a histogram of the top 12 key bits over the segment's part of the row, restricted to keys at or above
-//       a lower bound `lo` (a hint: the sampled cutoff, or the bin edge near last round's 3 k_s-th largest key), so
-//       that nearly all entries cost a compare and no shared-memory atomic.  From the top down, the bin b0 that
+//       a lower bound `lo` (a hint: the sampled cutoff, or in layer-wise mode the bound that the segment's last
+//       selection left: the key of the entry max(2 k_s, 32) places below its threshold), so that nearly all
+//       entries cost a compare and no shared-memory atomic.  From the top down, the bin b0 that
 //       holds the k_s-th largest, the entries above it and the number c0 inside it.  If the histogram holds
 //       fewer than k_s entries the hint was too high and the pass is repeated for that segment with lo an octave
 //       lower, and if need be a third time with lo = 0.
 //   (B) a second pass over the rows: entries above bin b0 are winners (mask bit set, composite appended to
 //       the worker's winner list); the c0 entries inside it go to a list of their own,
 //   (C) from which one block takes the `need` largest composites (key, lowest index).
+// In layer-wise mode the streaming pass has already gathered every entry at or above its segment's bound into the
+// worker's candidate list; (A) and (B) of such a segment read that list instead of the rows.
 // A segment whose bin b0 does not fit the list space (error feedback has packed thousands of entries into it, or
 // the row is full of equal values) stays on the rows for a second digit of 12 bits.  If its bin, 4096 times
 // narrower, fits, the segment goes the list way from there ((B) and (C) with 24 bits fixed).  Otherwise a third
@@ -1624,7 +1627,7 @@ struct DenseArgs {
   const int64_t* seg_tile0; // [n_seg + 1] first tile of each segment
   u32* dhist;               // [N][n_seg][kBins], all zero between launches
   SegState* seg;            // [N][n_seg]
-  u32* seg_thr;             // [N][n_seg] the lower bound the last round left for this one (a bin edge near its 3k-th largest key; 0: none)
+  u32* seg_thr;             // [N][n_seg] the lower bound the last round left for this one (see leave_rank_bound; 0: none)
   u32* tile_ties;           // [N][tiles][2]: entries equal to the threshold key in the tile, and in lower tiles of the segment
 };
 
