@@ -1979,7 +1979,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
           const SegState sg = load_seg(a, n, s);
           return sg.mode == want_mode ? (sg.lo | sg.src) : kFull;
         };
-        const int64_t gw = (int64_t)blockIdx.x * kDenseWarps + warp, nwarps = (int64_t)gridDim.x * kDenseWarps;
+        const int64_t gw = (int64_t)warp * gridDim.x + blockIdx.x, nwarps = (int64_t)gridDim.x * kDenseWarps;  // warps numbered across the blocks: a short run of tasks spreads over all SMs
         {  // candidates
           const int64_t tasks = s_cbase[nf];
           const int64_t per = (tasks + nwarps - 1) / nwarps;
@@ -2131,7 +2131,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
     // the rows and takes nothing from those after it.
     auto find_first = [&](int attempt) {
       const int64_t nwarps = (int64_t)gridDim.x * kDenseWarps;
-      for (int64_t v = (int64_t)blockIdx.x * kDenseWarps + warp; v < nsegs; v += nwarps) {
+      for (int64_t v = (int64_t)warp * gridDim.x + blockIdx.x; v < nsegs; v += nwarps) {  // (warps numbered across the blocks)
         const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
         const SegState old = load_seg(a, n, s);
         SegState* st = a.seg + (size_t)n * a.n_seg + s;
@@ -2457,7 +2457,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             if (cntA >= (u32)(kWarpList - 32)) flush_L();
           }
         };
-        const int64_t gw = (int64_t)blockIdx.x * kDenseWarps + warp, nwarps = (int64_t)gridDim.x * kDenseWarps;
+        const int64_t gw = (int64_t)warp * gridDim.x + blockIdx.x, nwarps = (int64_t)gridDim.x * kDenseWarps;  // warps numbered across the blocks: a short run of tasks spreads over all SMs
         {  // candidates
           const int64_t tasks = s_cbase[nf];
           const int64_t per = (tasks + nwarps - 1) / nwarps;
@@ -2935,7 +2935,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       const int nw = blockDim.x >> 5;
       const int64_t U = p.W >> 3;
       const int64_t seg_units = (U + a.emit_segments - 1) / a.emit_segments;
-      for (int64_t it = (int64_t)blockIdx.x * nw + warp; it < nf * a.emit_segments; it += (int64_t)gridDim.x * nw)
+      for (int64_t it = (int64_t)warp * gridDim.x + blockIdx.x; it < nf * a.emit_segments; it += (int64_t)gridDim.x * nw)  // (warps numbered across the blocks)
         post_prefix_segment(p, (int)s_flagged[it / a.emit_segments], (u32)(it % a.emit_segments), seg_units, lane);
       grid.sync();
       u32* s_segbase = s_hist;
