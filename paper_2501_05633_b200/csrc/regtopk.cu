@@ -2506,6 +2506,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
           }
         }
         flush_L();
+        __syncthreads();  // the tables in shared memory are free again: a histogram pass may follow at once
         return;
       }
       auto flush_A2 = [&](int n) {
@@ -2570,7 +2571,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
     // the first digit's search left stands.
     auto bound_rank = [&](const SegState& sg, int s) -> u32 {
       const u32 ks = (u32)(a.seg_kpre[s + 1] - a.seg_kpre[s]);
-      const u32 more = ks > 16u ? (ks > kFull / 4u ? kFull / 2u : 2u * ks) : 32u;
+      const u32 more = ks > 32u ? (ks > kFull / 4u ? kFull / 2u : ks) : 32u;
       return sg.need + more < more ? kFull : sg.need + more;
     };
     auto leave_rank_bound = [&](int n, int s, const SegState& sg, u32 key_r) {  // one thread

@@ -370,6 +370,20 @@ def test_layerwise_more_segments_than_the_shared_tables_hold(N, n_layers):
     run_parity(_drift_rounds(N, d, 5, seed=N, scales={}), d, N, 0, 4.0, layers=_layers_of(sizes, 0.1), threads=8)
 
 
+def test_layerwise_a_crowded_layer_beside_list_fed_ones():
+    """One layer of equal values (its threshold bin never fits the list space: second and third digit on the rows, ties
+    in index order) in a worker whose other layers are selected from the candidate list in the same launch."""
+    sizes = [30_000, 200_000, 64, 50_000, 20_011]
+    d = int(sum(sizes))
+    g = torch.Generator().manual_seed(41)
+    rounds = []
+    for t in range(8):
+        x = torch.randn((3, d), generator=g)
+        x[:, 30_000:230_000] = 0.25 if t % 2 == 0 else -0.125  # the crowded layer
+        rounds.append(x)
+    run_parity(rounds, d, 3, 0, 4.0, layers=_layers_of(sizes, 0.005), threads=8)
+
+
 def test_layerwise_sixty_rounds_on_a_tensor_table():
     """Long enough for the bounds that each layer's selection leaves for the next round to settle and to be missed now
     and then (ResNet-18's tensor table scaled down, error feedback ageing over 60 rounds)."""
