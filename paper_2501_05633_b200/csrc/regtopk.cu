@@ -1568,7 +1568,7 @@ __global__ void __launch_bounds__(256) k_unzip(UnzipArgs p) {
 // Per segment:
 //   (A) a histogram of the top 12 key bits over the segment's part of the row, restricted to keys at or above
 //       a lower bound `lo` (a hint: the sampled cutoff, or in layer-wise mode the bound that the segment's last
-//       selection left: the key of the entry max(2 k_s, 32) places below its threshold), so that nearly all
+//       selection left: the key of the entry max(k_s, 32) places below its threshold), so that nearly all
 //       entries cost a compare and no shared-memory atomic.  From the top down, the bin b0 that
 //       holds the k_s-th largest, the entries above it and the number c0 inside it.  If the histogram holds
 //       fewer than k_s entries the hint was too high and the pass is repeated for that segment with lo an octave
@@ -2565,7 +2565,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
     // ---- (C) per list segment: the `need` largest composites of its in-bin list win ----
     // Layer-wise mode: the lower bound a list segment leaves for the next round.  Error feedback packs more and more
     // entries right under the threshold, so the bound goes by rank, not by magnitude: it is the key of the entry
-    // max(2 k_s, 32) places below the threshold in the segment's in-bin list (bound_rank: its place in that list).
+    // max(k_s, 32) places below the threshold in the segment's in-bin list (bound_rank: its place in that list).
     // A list too short for that (few entries at or above this round's bound) widens the gap between the bound and
     // the threshold key by a half, as long as the bound lies inside the threshold's bin; otherwise the bin edge that
     // the first digit's search left stands.
