@@ -1596,7 +1596,8 @@ constexpr u32 kOctave = 0x00800000u;  // one binary order of magnitude in key un
 constexpr u32 kHintMargin = 2u << 19;  // two bins of the first digit (an eighth of an octave)
 
 enum : u32 { kSegList = 0u, kSegRows = 1u, kSegRetry = 2u, kSegList2 = 3u,
-             kSegWant = 4u };  // first digit found, list space not yet dealt out (only inside the first-digit search)
+             kSegWant = 4u,    // first digit found, list space not yet dealt out (only inside the first-digit search)
+             kSegZero = 5u };  // every key of the segment is zero (a layer without gradient): its lowest k_s indices win
 enum : u32 { kFlagRetry = 1u, kFlagRows = 2u, kFlagOrdered = 4u, kFlagBad = 8u, kFlagRows2 = 16u,
             kFlagWalk = 32u };  // layer-wise mode: some segment takes its first digit from the rows (otherwise no block walks its tiles for it)
 
@@ -1611,7 +1612,8 @@ struct __align__(16) SegState {
   u32 sh;      // key bits below the digits in `prefix` (19 after the first digit, 7 after the second)
   u32 src;     // 1: the first digit and the compaction read the worker's candidate list (layer-wise mode: the streaming
                //    pass gathered every entry at or above the segment's bound); 0: they walk the rows
-  u32 pad[3];
+  u32 nonzero; // set by the first digit's walk when it saw a key other than zero (or did not look: a bound was set)
+  u32 pad[2];
 };
 
 struct DenseArgs {
@@ -1743,7 +1745,7 @@ __device__ __forceinline__ SegState load_seg(const DenseArgs& a, int n, int s) {
   SegState r;
   r.prefix = v.x; r.need = v.y; r.ties = v.z; r.mode = v.w;
   r.lo = x.x; r.boff = x.y; r.bfill = x.z; r.sh = x.w;
-  r.src = y.x; r.pad[0] = r.pad[1] = r.pad[2] = 0u;
+  r.src = y.x; r.nonzero = y.y; r.pad[0] = r.pad[1] = 0u;
   return r;
 }
 
@@ -1843,7 +1845,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
   __shared__ u32 s_cbase[kDenseMaxFlagged + 1];  // layer-wise mode: 32-entry pieces of the candidate lists before each flagged worker's
   __shared__ u32 s_scan[33];
   __shared__ u32 s_res[4];
-  __shared__ u32 s_cnt, s_nf, s_nf2;
+  __shared__ u32 s_cnt, s_nf, s_nf2, s_nz;
   __shared__ u64 s_T;
   __shared__ u32 s_wcnt[1][kDenseWarps];
   cg::grid_group grid = cg::this_grid();
@@ -1908,6 +1910,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       SegState st;
       st.mode = ~0u;
       for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
+      if (tid == 0) s_nz = 0u;
       __syncthreads();
       for (int64_t w = walk ? w_begin : w_end; w < w_end; ++w) {
         const DenseTile t = dense_tile(a, s_flagged, w);
@@ -1915,13 +1918,16 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
           if (dirty) {
             __syncthreads();
             flush_hist(s_hist, a.dhist + ((size_t)cur_n * a.n_seg + cur_s) * kBins, kBins);
+            if (lv == 0 && tid == 0 && s_nz) atomicOr(&a.seg[(size_t)cur_n * a.n_seg + cur_s].nonzero, 1u);
             __syncthreads();
             for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
+            if (tid == 0) s_nz = 0u;
             __syncthreads();
             dirty = false;
           }
           cur_n = t.n; cur_s = t.s;
           st = load_seg(a, t.n, t.s);  // nothing writes it during this pass
+          if (lv == 0 && tid == 0 && st.lo != 0u) s_nz = 1u;  // a bound: the walk does not look at every entry, so the segment is not known to be all zero
         }
         if (st.mode != want_mode || (LAYERED && lv == 0 && st.src)) { w += a.seg_tile0[t.s + 1] - 1 - t.t; continue; }  // nothing to do in this segment: on to its last tile (the same in every thread of the block)
         dirty = true;
@@ -1942,13 +1948,22 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
               if (in[q] && key[q] >= st.lo) atomicAdd(&s_hist[key[q] >> 19], 1u);
           });
         } else if (lv == 0) {
-          dense_walk<true>(p, t.n, t.t0, t.t1, floor_key, count);  // (the previous support is counted from the override list)
+          u32 seen = 0;  // (the previous support is counted from the override list; its scores are zero where |a| is)
+          dense_walk<true>(p, t.n, t.t0, t.t1, floor_key, [&](int64_t j4, const u32 (&key)[4], const bool (&in)[4]) {
+            count(j4, key, in);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) seen |= in[q] ? key[q] : 0u;
+          });
+          if (seen) s_nz = 1u;
         } else {
           dense_walk<false>(p, t.n, t.t0, t.t1, floor_key, count);
         }
       }
       __syncthreads();
-      if (dirty) flush_hist(s_hist, a.dhist + ((size_t)cur_n * a.n_seg + cur_s) * kBins, kBins);
+      if (dirty) {
+        flush_hist(s_hist, a.dhist + ((size_t)cur_n * a.n_seg + cur_s) * kBins, kBins);
+        if (lv == 0 && tid == 0 && s_nz) atomicOr(&a.seg[(size_t)cur_n * a.n_seg + cur_s].nonzero, 1u);
+      }
       if (LAYERED && lv == 0) {
         // Layer-wise mode: the candidate lists of the segments fed from them, and the entries of the previous
         // support (override list), as one run of 32-entry tasks over all flagged workers, dealt to the warps of the
@@ -2193,7 +2208,12 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             }
             cum += __shfl_sync(kFull, incl, 31);
           }
-          if (lane == 0) {
+          if (lane == 0 && !old.src && old.lo == 0u && !old.nonzero) {
+            // the walk looked at every entry and saw no key but zero (scores on the previous support are zero where
+            // the accumulator is): the segment's lowest k_s indices win; nothing to search, no list, no bound
+            st->mode = kSegZero; st->prefix = 0; st->need = need; st->ties = 0;
+            a.seg_thr[(size_t)n * a.n_seg + s] = 0u;
+          } else if (lane == 0) {
             if (b == kFull) {
               if (old.lo == 0u) {  // fewer than k entries in the whole segment: cannot happen
                 atomicOr(&p.gctl->dense_flags, kFlagBad);
@@ -2292,7 +2312,8 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       // gather by or the list overflowed
       st.src = (LAYERED && lo != 0u && (u64)p.ctl[n].cand_count <= (u64)p.capA) ? 1u : 0u;
       if (LAYERED && !st.src) atomicOr(&p.gctl->dense_flags, kFlagWalk);
-      st.pad[0] = st.pad[1] = st.pad[2] = 0u;
+      st.nonzero = 0u;
+      st.pad[0] = st.pad[1] = 0u;
       a.seg[(size_t)n * a.n_seg + s] = st;
     }
     grid.sync();
@@ -2590,9 +2611,21 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
      for (int64_t v = blockIdx.x; v < nsegs; v += gridDim.x) {
       const int n = (int)s_flagged[v / a.n_seg], s = (int)(v % a.n_seg);
       const SegState st = load_seg(a, n, s);
+      u32* mask = p.mask_new + (size_t)n * p.W;
+      if (want_mode == kSegList && st.mode == kSegZero) {  // an all-zero segment: its first k_s coordinates
+        __syncthreads();
+        if (tid == 0) s_cnt = atomicAdd(&p.ctl[n].acount, st.need);
+        __syncthreads();
+        const u32 first = (u32)(s ? a.seg_end[s - 1] : 0);
+        for (u32 i = tid; i < st.need; i += blockDim.x) {
+          set_winner(mask, first + i, p.d);
+          if (RT_INB((u64)s_cnt + i < (u64)k)) p.ovr_comp[(size_t)n * p.k + s_cnt + i] = make_composite(0u, first + i);
+        }
+        __syncthreads();
+        continue;
+      }
       if (st.mode != want_mode || st.need == 0u) continue;  // the same in every thread of the block
       const u64* list = p.candB + (size_t)n * p.stride + st.boff;
-      u32* mask = p.mask_new + (size_t)n * p.W;
       const u32 count = st.ties;
       if (st.bfill != count) {
         if (tid == 0) atomicOr(&p.gctl->dense_flags, kFlagBad);
