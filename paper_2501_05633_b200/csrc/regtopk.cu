@@ -1878,6 +1878,11 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
     const int64_t w_begin = (int64_t)blockIdx.x * per < total_tiles ? (int64_t)blockIdx.x * per : total_tiles;
     const int64_t w_end = w_begin + per < total_tiles ? w_begin + per : total_tiles;
     const int64_t nsegs = nf * a.n_seg;
+    // The two walks of the first digit take the tiles in runs: one contiguous run per block in the plain mode; in
+    // layer-wise mode runs of 16 tiles dealt round-robin, because there the tiles to be walked (layers without a bound,
+    // layers without gradient) lie in clusters that contiguous runs would leave to a few blocks.
+    const int64_t t_run = LAYERED ? 16 : per;
+    const int64_t t_step = LAYERED ? (int64_t)gridDim.x * 16 : (total_tiles > 0 ? total_tiles : 1);
     if (LAYERED) {  // (a worker whose list overflowed has no pieces: none of its segments is fed from the list)
       constexpr int kPer = kDenseMaxFlagged / kDenseThreads;
       u32 mine[kPer], sum = 0, total;
@@ -1912,13 +1917,15 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
       if (tid == 0) s_nz = 0u;
       __syncthreads();
-      for (int64_t w = walk ? w_begin : w_end; w < w_end; ++w) {
+      for (int64_t c0 = walk ? (int64_t)blockIdx.x * t_run : total_tiles; c0 < total_tiles; c0 += t_step)
+      for (int64_t w = c0, c1 = c0 + t_run < total_tiles ? c0 + t_run : total_tiles; w < c1; ++w) {
         const DenseTile t = dense_tile(a, s_flagged, w);
         if (t.n != cur_n || t.s != cur_s) {
           if (dirty) {
             __syncthreads();
             flush_hist(s_hist, a.dhist + ((size_t)cur_n * a.n_seg + cur_s) * kBins, kBins);
-            if (lv == 0 && tid == 0 && s_nz) atomicOr(&a.seg[(size_t)cur_n * a.n_seg + cur_s].nonzero, 1u);
+            // (with a bound the walk did not look at every entry: the segment is not known to be all zero)
+            if (lv == 0 && tid == 0 && (s_nz || st.lo != 0u)) atomicOr(&a.seg[(size_t)cur_n * a.n_seg + cur_s].nonzero, 1u);
             __syncthreads();
             for (int i = tid; i < kBins; i += blockDim.x) s_hist[i] = 0;
             if (tid == 0) s_nz = 0u;
@@ -1927,7 +1934,6 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
           }
           cur_n = t.n; cur_s = t.s;
           st = load_seg(a, t.n, t.s);  // nothing writes it during this pass
-          if (lv == 0 && tid == 0 && st.lo != 0u) s_nz = 1u;  // a bound: the walk does not look at every entry, so the segment is not known to be all zero
         }
         if (st.mode != want_mode || (LAYERED && lv == 0 && st.src)) { w += a.seg_tile0[t.s + 1] - 1 - t.t; continue; }  // nothing to do in this segment: on to its last tile (the same in every thread of the block)
         dirty = true;
@@ -1950,7 +1956,14 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         } else if (lv == 0) {
           u32 seen = 0;  // (the previous support is counted from the override list; its scores are zero where |a| is)
           dense_walk<true>(p, t.n, t.t0, t.t1, floor_key, [&](int64_t j4, const u32 (&key)[4], const bool (&in)[4]) {
-            count(j4, key, in);
+            // 128 equal keys (a stretch without gradient) are counted with one addition
+            const u32 v = __shfl_sync(kFull, key[0], 0);
+            const bool same = in[0] && in[1] && in[2] && in[3] && key[0] == v && key[1] == v && key[2] == v && key[3] == v;
+            if (__all_sync(kFull, same)) {
+              if (lane == 0) atomicAdd(&s_hist[v >> 19], 128u);
+            } else {
+              count(j4, key, in);
+            }
 #pragma unroll
             for (int q = 0; q < 4; ++q) seen |= in[q] ? key[q] : 0u;
           });
@@ -1962,7 +1975,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       __syncthreads();
       if (dirty) {
         flush_hist(s_hist, a.dhist + ((size_t)cur_n * a.n_seg + cur_s) * kBins, kBins);
-        if (lv == 0 && tid == 0 && s_nz) atomicOr(&a.seg[(size_t)cur_n * a.n_seg + cur_s].nonzero, 1u);
+        if (lv == 0 && tid == 0 && (s_nz || st.lo != 0u)) atomicOr(&a.seg[(size_t)cur_n * a.n_seg + cur_s].nonzero, 1u);
       }
       if (LAYERED && lv == 0) {
         // Layer-wise mode: the candidate lists of the segments fed from them, and the entries of the previous
@@ -2389,7 +2402,8 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       __syncwarp();
       SegState st;
       st.mode = ~0u;
-      for (int64_t w = walk ? w_begin : w_end; w < w_end; ++w) {
+      for (int64_t c0 = walk ? (int64_t)blockIdx.x * t_run : total_tiles; c0 < total_tiles; c0 += t_step)
+      for (int64_t w = c0, c1 = c0 + t_run < total_tiles ? c0 + t_run : total_tiles; w < c1; ++w) {
         const DenseTile t = dense_tile(a, s_flagged, w);
         if (t.n != cur_n || t.s != cur_s) {
           if (cur_n >= 0 && st.mode == want_mode) flush(cur_n, cur_s, st);
