@@ -2140,10 +2140,14 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         __syncthreads();
         block_find_from_top(s_hist, kBins, need, s_scan, s_res);
         const u32 b = s_res[0], above = s_res[1];
-        u32 b_wide = kFull;  // first digit only: the bin of the entry three times as far down, for the next round's bound
-        if (lv == 0 && b != kFull) {
+        // for the next round's bound: the bin of the entry three times as far down (first digit); in layer-wise mode,
+        // after the second digit, the sub-bin of the entry max(k_s, 32) places below the threshold
+        u32 b_wide = kFull;
+        const u32 ks_seg = (u32)(a.seg_kpre[s + 1] - a.seg_kpre[s]);
+        const u32 r2 = lv == 0 ? 3u * need : ((LAYERED && lv == 1) ? need + (ks_seg > 32u ? ks_seg : 32u) : 0u);
+        if (r2 > need && b != kFull) {
           __syncthreads();
-          block_find_from_top(s_hist, kBins, 3u * need, s_scan, s_res);
+          block_find_from_top(s_hist, kBins, r2, s_scan, s_res);
           b_wide = s_res[0];
         }
         if (tid == 0) done(n, s, old, need, b, above, b == kFull ? 0u : s_hist[b], b_wide);
@@ -2831,9 +2835,12 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
       // Second digit of the segments whose first bin was too crowded for the list space.  After it the bin is 4096
       // times narrower: if it fits now, the segment goes the list way from here (one more pass over the rows);
       // otherwise (rows of equal keys) the third digit and the ordered take of ties follow.
-      find_pass(1, kSegRows, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin, u32) {
+      find_pass(1, kSegRows, [&](int n, int s, const SegState& old, u32 need, u32 b, u32 above, u32 in_bin, u32 b_rank) {
         SegState* st = a.seg + (size_t)n * a.n_seg + s;
         if (b == kFull) { atomicOr(&p.gctl->dense_flags, kFlagBad); b = 0; above = 0; }
+        // (layer-wise mode) a bound by rank for the next round, as the list segments leave one: without it the bin edge
+        // from the first digit stands, a sixteenth of an octave wide, and the next candidate list overflows
+        if (LAYERED && b_rank != kFull) a.seg_thr[(size_t)n * a.n_seg + s] = (((old.prefix << 12) | b_rank) << 7) & ~1u;
         st->prefix = (old.prefix << 12) | b;
         st->need = need - above;
         st->ties = in_bin;
