@@ -829,6 +829,15 @@ def test_full_size_layerwise_resnet18():
     run_parity((s.next() for _ in range(10)), w.d, w.N, 0, w.mu, layers=L, threads=8)
 
 
+def test_full_size_layerwise_resnet50():
+    """The ResNet-50 table at full size: 30 % of its coordinates lie in frozen tensors (no gradient), whose layers select
+    their lowest indices; one tensor is frozen in part."""
+    w = synth.workload("resnet50")
+    L = _layers_of(w.shapes, w.sparsity[0])
+    s = synth.GradientStream(w, device="cuda", seed=0, pad_to=32)
+    run_parity((s.next() for _ in range(4)), w.d, w.N, 0, w.mu, layers=L, threads=8)
+
+
 def test_full_size_layerwise_certified_gpt2():
     """The GPT-2 table (bf16 gradients, 148 layers with 0.01 % each) at full size, certified layer by layer without a
     sort: inside every layer no entry outside the library's selection ranks before its last-ranked entry."""
