@@ -1983,13 +1983,13 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         // grid in contiguous pieces.  The segment ends and the segments' bounds are looked up in shared memory
         // (the staging space, not used in this pass) when they fit there.
         u32* t_end = reinterpret_cast<u32*>(s_stage);  // [n_seg]
-        u32* t_lo = t_end + a.n_seg;                   // [nsegs]: bound | list-fed, or kFull if the segment takes no part
+        u32* t_lo = t_end + a.n_seg;                   // [nsegs]: bound (keys have 31 bits) | list-fed << 31, or kFull if the segment takes no part
         const bool fast = (u64)nsegs + (u64)a.n_seg <= (u64)kDenseWarps * 2u * kWarpList * 2u;
         if (fast) {
           for (int i = tid; i < a.n_seg; i += blockDim.x) t_end[i] = (u32)a.seg_end[i];
           for (int64_t v = tid; v < nsegs; v += blockDim.x) {
             const SegState sg = load_seg(a, (int)s_flagged[v / a.n_seg], (int)(v % a.n_seg));
-            t_lo[v] = sg.mode == want_mode ? (sg.lo | sg.src) : kFull;
+            t_lo[v] = sg.mode == want_mode ? (sg.lo | (sg.src << 31)) : kFull;
           }
           __syncthreads();
         }
@@ -2005,7 +2005,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
         auto bound_of = [&](int64_t f, int n, int s) -> u32 {
           if (fast) return t_lo[f * a.n_seg + s];
           const SegState sg = load_seg(a, n, s);
-          return sg.mode == want_mode ? (sg.lo | sg.src) : kFull;
+          return sg.mode == want_mode ? (sg.lo | (sg.src << 31)) : kFull;
         };
         const int64_t gw = (int64_t)warp * gridDim.x + blockIdx.x, nwarps = (int64_t)gridDim.x * kDenseWarps;  // warps numbered across the blocks: a short run of tasks spreads over all SMs
         {  // candidates
@@ -2042,7 +2042,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             const u32 key = (u32)(c >> 32);
             const int s = (live && a.n_seg > 1) ? seg_of(composite_idx(c)) : 0;
             const u32 bound = live ? bound_of(f, n, s) : kFull;
-            const bool use = bound != kFull && (bound & 1u) && key >= (bound & ~1u);
+            const bool use = bound != kFull && (bound >> 31) && key >= (bound & 0x7FFFFFFFu);
             u32* target = a.dhist + ((size_t)n * a.n_seg + s) * kBins + (key >> 19);
             const u32 act = __ballot_sync(kFull, use);
             if (use) {
@@ -2065,7 +2065,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             const int s = (live && a.n_seg > 1) ? seg_of((u32)j) : 0;
             const u32 bound = live ? bound_of(f, n, s) : kFull;
             const bool part = bound != kFull;
-            const u32 lo_seg = bound & ~1u;
+            const u32 lo_seg = bound & 0x7FFFFFFFu;
             const bool use = part && key >= lo_seg;
             u32* hist = a.dhist + ((size_t)n * a.n_seg + s) * kBins;
             u32* target = hist + (key >> 19);
@@ -2076,7 +2076,7 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             }
             // a segment counted from the rows has the entry under bits(|a|): take that back (a list-fed one never
             // counted it: the list has no entries of the previous support)
-            if (part && !(bound & 1u)) {
+            if (part && !(bound >> 31)) {
               const u32 ka = __float_as_uint(p.eps[(size_t)n * p.ld + j]) & 0x7FFFFFFFu;
               if (ka >= lo_seg) atomicSub(hist + (ka >> 19), 1u);
             }
@@ -2229,7 +2229,14 @@ __global__ void __launch_bounds__(kDenseThreads, 2) k_dense(DenseArgs a) {
             // the walk looked at every entry and saw no key but zero (scores on the previous support are zero where
             // the accumulator is): the segment's lowest k_s indices win; nothing to search, no list, no bound
             st->mode = kSegZero; st->prefix = 0; st->need = need; st->ties = 0;
-            a.seg_thr[(size_t)n * a.n_seg + s] = 0u;
+            // layer-wise mode: the bound 1 for the next round: the streaming pass then gathers every entry of the layer
+            // that is not zero, and a layer that sends none is known to be all zero without a walk
+            a.seg_thr[(size_t)n * a.n_seg + s] = LAYERED ? 1u : 0u;
+          } else if (lane == 0 && LAYERED && old.src && old.lo == 1u && cum == 0u) {
+            // the bound was 1 and the candidate list holds no entry of this segment (nor has the override list one
+            // with a score other than zero): every key is zero again
+            st->mode = kSegZero; st->prefix = 0; st->need = need; st->ties = 0;
+            a.seg_thr[(size_t)n * a.n_seg + s] = 1u;
           } else if (lane == 0) {
             if (b == kFull) {
               if (old.lo == 0u) {  // fewer than k entries in the whole segment: cannot happen
